@@ -1,0 +1,229 @@
+/*
+ * compass.h -- C ABI of the B200 (sm_100a) implementation of Compass's
+ * tensor-parallel hot path: fused AllGather+GEMM and GEMM+ReduceScatter whose
+ * tiles are visited in the order of the double-ring chunk schedule
+ * (TA-IntraFusion, Section III), the decomposed pipeline (ODP-InterDecom,
+ * Section IV) and the strategy selector (Algorithm 1, Section V).
+ *
+ * The tensor-parallel group is P logical ranks on ONE GPU: every rank's
+ * shards and outputs are separate device allocations, passed as arrays of P
+ * pointers.  All tensors are BF16, row-major, densely packed:
+ *
+ *   AllGather+GEMM   (Section II-A): rank r holds A_r [M/P x K] and the
+ *       weight shard B_r stored K-major as [N x K] (N = columns PER RANK);
+ *       the call produces C_r [M x N] = [A_0; ...; A_{P-1}] * B_r^T for all r.
+ *   GEMM+ReduceScatter (Section II-A): rank r holds A_r [M x K] (K = PER-RANK
+ *       slice of the contraction) and B_r [N x K]; the call produces
+ *       Out_r [M/P x N] = rows [r*M/P, (r+1)*M/P) of sum_q A_q * B_q^T.
+ *
+ * Accumulation is FP32, outputs are rounded once to BF16 (round to nearest
+ * even) unless a variant says otherwise.
+ *
+ * Ownership and errors.  The caller owns every buffer, including the
+ * workspace; the library allocates no device memory.  Pointer arrays live in
+ * host memory and are read before the call returns; the tensors they point to
+ * are device memory unless an entry point says "host".  Device work is
+ * asynchronous on the caller's stream(s).  Inputs are never written.  Every
+ * function returns a compass_status; nothing throws, aborts or traps.
+ * Arguments are checked on the host before any launch.  Device-side waits are
+ * bounded: a wait that gives up records COMPASS_ERR_TIMEOUT in the status
+ * block at the start of the workspace (see compass_read_status).
+ */
+#ifndef COMPASS_H
+#define COMPASS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define COMPASS_MAX_P 16            /* largest tensor-parallel size accepted */
+#define COMPASS_STATUS_BYTES 256    /* status block at the start of every workspace */
+
+typedef enum compass_status {
+  COMPASS_OK = 0,
+  COMPASS_ERR_INVALID_ARG = 1,      /* NULL pointer, P < 1, rings not 1|2, d < 1, unknown op/variant */
+  COMPASS_ERR_SHAPE = 2,            /* M % P, (M/P) % rings, (M/P) % d non-zero; M, N or K <= 0 */
+  COMPASS_ERR_UNSUPPORTED = 3,      /* dtype other than BF16, P > COMPASS_MAX_P, sizes beyond int32 rows */
+  COMPASS_ERR_ALIGNMENT = 4,        /* a tensor pointer not 16-byte aligned, or K % 8 / N % 8 non-zero
+                                       (rows must be a multiple of 16 bytes for the tensor-map loads) */
+  COMPASS_ERR_BUFFER_TOO_SMALL = 5, /* schedule capacity or workspace bytes */
+  COMPASS_ERR_CUDA = 6,             /* a CUDA call failed; see compass_last_cuda_error() */
+  COMPASS_ERR_TIMEOUT = 7           /* a bounded device-side wait gave up (from compass_read_status) */
+} compass_status;
+
+enum { COMPASS_OP_AG_GEMM = 0, COMPASS_OP_GEMM_RS = 1 };
+enum { COMPASS_DTYPE_BF16 = 0 };
+/* GEMM+ReduceScatter variants.
+ *   SEGMENTED_K: an output tile's accumulator runs over the P ranks' K-slices
+ *     in ring order (the reduction tree is the tensor-core accumulator); one
+ *     BF16 rounding.
+ *   RING_RMW: every rank's partial tile is produced separately in that rank's
+ *     schedule order and added into the owner's rows in ring order by a
+ *     vectorised read-modify-write in the GEMM epilogue (the running sum is
+ *     kept in FP32 in the workspace; the owner's contribution, scheduled last,
+ *     writes the BF16 result).  Needs tile counters in the workspace. */
+enum { COMPASS_RS_SEGMENTED_K = 0, COMPASS_RS_RING_RMW = 1 };
+enum { COMPASS_STRATEGY_INTRAFUSION = 0, COMPASS_STRATEGY_INTERDECOM = 1 };
+/* selectors for compass_workspace_bytes */
+enum { COMPASS_WS_FUSED = 0, COMPASS_WS_DECOMP = 1 };
+
+/* Workload descriptor W = (pattern, M, N, K, world size[, d]) of Table IV and
+ * Algorithm 1.  See the header comment for the meaning of M, N, K per op. */
+typedef struct compass_problem {
+  int32_t op;          /* COMPASS_OP_* */
+  int32_t P;           /* tensor-parallel size, 1..COMPASS_MAX_P */
+  int32_t rings;       /* 2 = double ring (default of the paper inside a NUMA domain), 1 = single ring */
+  int32_t d;           /* decomposition degree for compass_decomp (>= 1); ignored elsewhere */
+  int64_t M, N, K;
+  int32_t dtype;       /* COMPASS_DTYPE_BF16 */
+  int32_t rs_variant;  /* COMPASS_RS_* (GEMM+ReduceScatter only) */
+} compass_problem;
+
+/* One line of the ring chunk schedule (Section III-B).  `part` = rings*chunk +
+ * ring; with two rings ring 0 is the backward ring (r -> r-1, even partitions,
+ * first half of a chunk's rows) and ring 1 the forward ring (r -> r+1, odd
+ * partitions, second half); a single ring is the forward ring.  `peer` is the
+ * neighbour the partition arrives from (AllGather) or is sent to
+ * (ReduceScatter) and equals `rank` for the local entry.  row_begin/row_count
+ * address rows of the gathered (AG) or fully reduced (RS) tensor. */
+typedef struct compass_sched_entry {
+  int32_t rank, step, ring, part, chunk, peer, row_begin, row_count;
+} compass_sched_entry;
+
+/* Calibrated parameters (Section IV-C, V-B; Algorithm 1 phase 2) for ONE
+ * pattern: T_comp = comp_a + comp_b*FLOPs, T_comm = comm_a + comm_b*bytes with
+ * FLOPs = 2*P*M*N*K and bytes = 2*P*M*K (AG) or 2*P*M*N (RS); eta(d) =
+ * alpha_decomp + beta_decomp*d (Eq. 3); fusion overhead per synchronisation
+ * point alpha_fusion + beta_fusion*m (Eq. 8).  Times in any one unit. */
+typedef struct compass_calib {
+  double comp_a, comp_b, comm_a, comm_b;
+  double alpha_decomp, beta_decomp, alpha_fusion, beta_fusion;
+} compass_calib;
+
+typedef struct compass_choice {
+  int32_t strategy;    /* COMPASS_STRATEGY_* */
+  int32_t d_star;      /* Eq. 4-5 */
+  double t_fusion;     /* Eq. 7 */
+  double t_decomp;     /* Eq. 2 at d_star */
+  double t_comp, t_comm, lambda;
+  double t_star;       /* min(t_fusion, t_decomp) */
+} compass_choice;
+
+/* One block of a fused launch, in launch order (a diagnostic view of how a
+ * call maps the schedule onto the kernel; see compass_launch_plan). */
+typedef struct compass_plan_block {
+  int32_t rank, step, ring, part;      /* schedule entry this block executes (rank = -1: shared by all) */
+  int32_t a_tensor, a_row_begin;       /* which A pointer is read, first row inside it */
+  int32_t out_tensor, out_row_begin;   /* which output pointer is written, first row inside it */
+  int32_t rows;
+  int32_t first_tile, tile_count;      /* tiles [first_tile, first_tile+tile_count) of the launch */
+} compass_plan_block;
+
+/* ---- schedule (Section III-A, III-B) -------------------------------------
+ * Emits the ring chunk order: for every rank, P steps x `rings` entries;
+ * AllGather+GEMM processes the local chunk at step 0, GEMM+ReduceScatter at
+ * step P-1.  Order: rank-major, then step, then ring.  Writes rings*P*P
+ * entries to `out` (host memory) and the number to *count.  With out == NULL
+ * only *count is written.  Pure host integer code, deterministic. */
+int compass_schedule(int op, int P, int rings, int64_t M,
+                     compass_sched_entry* out, size_t capacity, size_t* count);
+
+/* ---- fused AllGather+GEMM (TA-IntraFusion, Section III-B) ----------------
+ * ONE kernel launch computes C_r for all ranks.  A tile of C_r that belongs
+ * to partition p of rank r's schedule reads its A rows directly from the
+ * shard of the rank that owns p (the gather is done by address, there is no
+ * gather buffer) and is issued in schedule order: step-major; inside a step
+ * ranks are interleaved per ring.
+ *   A: P device pointers, A[r] = [M/P x K];  B: P device pointers [N x K];
+ *   C: P device pointers [M x N] (every element is written).
+ *   workspace: >= compass_workspace_bytes(problem, COMPASS_WS_FUSED) bytes of
+ *   device memory, 256-byte aligned, whose status block was zeroed once with
+ *   compass_workspace_init.  cuda_stream: a cudaStream_t (NULL = default). */
+int compass_ag_gemm(const compass_problem* problem, const void* const* A, const void* const* B,
+                    void* const* C, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---- fused GEMM+ReduceScatter (Section III-B, last paragraph) ------------
+ * ONE kernel launch, no separate reduce kernel.  For partition p = (chunk c,
+ * ring g) the contributions are added in the order in which the running sum
+ * would travel the ring, ending with the owner c.
+ *   A: P device pointers [M x K];  B: P device pointers [N x K];
+ *   Out: P device pointers [M/P x N] (every element is written). */
+int compass_gemm_rs(const compass_problem* problem, const void* const* A, const void* const* B,
+                    void* const* Out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---- ODP-InterDecom (Section II-B, IV) -----------------------------------
+ * The same result as the fused calls, computed as problem->d sub-operators
+ * pipelined on two streams.  The operator is split along rows: with
+ * s = M/P/d, sub-operator j handles rows [j*s, (j+1)*s) of every chunk.
+ *   AG: sub-collective j = device-to-device copies of row slice j of every
+ *       shard into every rank's gather buffer (in the workspace) on
+ *       stream_copy; sub-GEMM j on stream_compute once they have landed.
+ *   RS: sub-GEMM j writes every rank's BF16 partial rows (workspace) on
+ *       stream_compute; sub-collective j = a reduce kernel on stream_copy
+ *       that sums the P partial slices in FP32 into the owners' rows.
+ * d = 1 is sequential execution.  On return all work is ordered before later
+ * work on stream_compute.  out = C (AG) or Out (RS) as in the fused calls.
+ * stream_copy must differ from stream_compute for overlap (equal is legal). */
+int compass_decomp(const compass_problem* problem, const void* const* A, const void* const* B,
+                   void* const* out, void* workspace, size_t workspace_bytes,
+                   void* stream_compute, void* stream_copy);
+
+/* ---- strategy selector (Algorithm 1) -------------------------------------
+ * Phase 1: T_comp, T_comm, lambda from the calibrated linear models; phase 2:
+ * d* by Eq. 4-5 (restricted to degrees that divide M/P); phase 3: T_decomp
+ * (Eq. 2) against T_fusion (Eq. 7-8); IntraFusion only if strictly faster.
+ * Host arithmetic only. */
+int compass_select(const compass_problem* problem, const compass_calib* calib, compass_choice* out);
+
+/* ---- models, individually (host) ----------------------------------------- */
+/* Eq. 2-3: (d-1)*max(T_comp,T_comm)/d*(alpha+beta*d) + T_comp/d + T_comm/d. */
+int compass_model_decomp_time(double t_comp, double t_comm, double alpha, double beta, int d, double* out);
+/* Eq. 4-5.  d_max: largest admissible degree (1..16).  as_printed != 0
+ * evaluates Eq. 5 literally with 1/lambda; 0 uses min(lambda, 1/lambda),
+ * which is the stationary point of Eq. 2 in both regimes.  *d_continuous
+ * (may be NULL) receives the argument of P_2, or -1 if it does not exist. */
+int compass_model_optimal_degree(double t_comp, double t_comm, double alpha, double beta, int d_max,
+                                 int as_printed, int* d_final, double* d_continuous);
+/* Eq. 7-8 with equal chunks: T_comp/n per chunk, T_comm/(n-1) per step. */
+int compass_model_fusion_time(double t_comp, double t_comm, int n_chunks, double alpha_f, double beta_f,
+                              double m_volume, double* out);
+/* One-time offline regressions (Section IV-C): eta measured at each sample
+ * (t_comp[i], t_comm[i], d[i] > 1, t_measured[i]) regressed on d. */
+int compass_calib_fit_decomp(const double* t_comp, const double* t_comm, const int* d, const double* t_measured,
+                             size_t n, double* alpha, double* beta);
+/* Residual of Eq. 7 per synchronisation point regressed on the message volume m. */
+int compass_calib_fit_fusion(const double* t_comp, const double* t_comm, const int* n_chunks, const double* m_volume,
+                             const double* t_measured, size_t n, double* alpha_f, double* beta_f);
+
+/* ---- helpers ------------------------------------------------------------- */
+/* Workspace size in bytes for the fused call (which = COMPASS_WS_FUSED) or for
+ * compass_decomp (COMPASS_WS_DECOMP) of this problem. */
+int compass_workspace_bytes(const compass_problem* problem, int which, size_t* bytes);
+/* Zero the status block and every counter of a workspace (asynchronous). */
+int compass_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream);
+/* Synchronise the stream and return the device-side status recorded in the
+ * workspace (COMPASS_OK or COMPASS_ERR_TIMEOUT); *detail (may be NULL) gets
+ * a code telling which wait gave up. */
+int compass_read_status(void* workspace, void* cuda_stream, int* detail);
+/* The blocks of the fused launch for this problem, in launch order. */
+int compass_launch_plan(const compass_problem* problem, compass_plan_block* out, size_t capacity, size_t* count);
+/* End-to-end convenience with HOST tensors: copies A and B (host pointers,
+ * pinned memory recommended) into `staging` (device, >= *staging_bytes_needed),
+ * runs the fused operator of problem->op and copies the outputs back to the
+ * host pointers in `out`; all asynchronous on cuda_stream.  With staging ==
+ * NULL only *staging_bytes_needed is written. */
+int compass_fused_host(const compass_problem* problem, const void* const* A_host, const void* const* B_host,
+                       void* const* out_host, void* staging, size_t staging_bytes, size_t* staging_bytes_needed,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+const char* compass_status_string(int status);
+int compass_last_cuda_error(void);
+/* Number of kernels this library has launched since it was loaded. */
+uint64_t compass_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COMPASS_H */

@@ -113,6 +113,8 @@ def d_candidate(t_comp: float, t_comm: float, alpha: float, beta: float,
             if decomp_time(t_comp, t_comm, alpha, beta, d) < decomp_time(t_comp, t_comm, alpha, beta, best):
                 best = d
         return best
+    if x >= 2.0 * cands[-1]:                 # also covers an overflowed (infinite) argument
+        return cands[-1]
     d = nearest_power_of_two(x)
     return min(max(d, cands[0]), cands[-1])
 

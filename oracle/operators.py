@@ -128,6 +128,37 @@ def gemm_rs(A: Sequence[np.ndarray], B: Sequence[np.ndarray], table: Optional[np
     return result
 
 
+def gemm_rs_rows(A: Sequence[np.ndarray], B: Sequence[np.ndarray], rows: np.ndarray,
+                 table: Optional[np.ndarray] = None, rings: int = 2):
+    """GEMM+ReduceScatter restricted to some rows of the reduced [M x N] tensor
+    (sorted global row indices), for sampling large cases.  Same ring order as
+    ``gemm_rs``.  Returns {owner chunk: (rows inside the owner's block, values)}."""
+    P = len(A)
+    M, K = A[0].shape
+    m = M // P
+    if table is None:
+        table = schedule(OP_GEMM_RS, P, rings, M)
+    rows = np.asarray(rows, dtype=np.int64)
+    Bf = [bf16_bits_to_f64(b) for b in B]
+    parts = {}
+    for e in table:
+        parts.setdefault(int(e[PART]), []).append(e)
+    found = {}
+    for part, entries in sorted(parts.items()):
+        entries = sorted(entries, key=lambda e: int(e[STEP]))
+        c, rb, rc = int(entries[0][CHUNK]), int(entries[0][ROW_BEGIN]), int(entries[0][ROW_COUNT])
+        sel = rows[(rows >= rb) & (rows < rb + rc)]
+        if sel.size == 0:
+            continue
+        running = np.zeros((sel.size, Bf[0].shape[0]))
+        for e in entries:
+            q = int(e[RANK])
+            running += bf16_bits_to_f64(A[q][sel]) @ Bf[q].T
+        assert int(entries[-1][RANK]) == c
+        found.setdefault(c, []).append((sel - c * m, running))
+    return {c: (np.concatenate([x[0] for x in v]), np.concatenate([x[1] for x in v])) for c, v in found.items()}
+
+
 def decomp_ag_gemm(A: Sequence[np.ndarray], B: Sequence[np.ndarray], d: int) -> List[np.ndarray]:
     """InterDecom of AllGather+GEMM into d sub-operators (Section II-B).
 

@@ -1,0 +1,506 @@
+// C ABI entry points: argument checks, mapping of the ring schedule onto GEMM
+// launches, the InterDecom stream pipeline, workspace layout.
+#include <atomic>
+#include <cstring>
+#include <mutex>
+
+#include "internal.h"
+
+namespace compass {
+
+namespace {
+
+std::atomic<int> g_last_cuda_error{0};
+std::atomic<uint64_t> g_kernel_launches{0};
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int validate_problem(const compass_problem* pr, int want_op, bool need_d) {
+  if (pr == nullptr) return COMPASS_ERR_INVALID_ARG;
+  if (pr->op != COMPASS_OP_AG_GEMM && pr->op != COMPASS_OP_GEMM_RS) return COMPASS_ERR_INVALID_ARG;
+  if (want_op >= 0 && pr->op != want_op) return COMPASS_ERR_INVALID_ARG;
+  if (pr->P < 1 || (pr->rings != 1 && pr->rings != 2)) return COMPASS_ERR_INVALID_ARG;
+  if (need_d && pr->d < 1) return COMPASS_ERR_INVALID_ARG;
+  if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant != COMPASS_RS_SEGMENTED_K && pr->rs_variant != COMPASS_RS_RING_RMW)
+    return COMPASS_ERR_INVALID_ARG;
+  if (pr->dtype != COMPASS_DTYPE_BF16 || pr->P > COMPASS_MAX_P) return COMPASS_ERR_UNSUPPORTED;
+  if (pr->M <= 0 || pr->N <= 0 || pr->K <= 0) return COMPASS_ERR_SHAPE;
+  if (pr->M % pr->P != 0 || (pr->M / pr->P) % pr->rings != 0) return COMPASS_ERR_SHAPE;
+  if (need_d && (pr->M / pr->P) % pr->d != 0) return COMPASS_ERR_SHAPE;
+  if (pr->K % 8 != 0 || pr->N % 8 != 0) return COMPASS_ERR_ALIGNMENT;
+  if (pr->M > (1 << 30) || pr->N > (1 << 30) || pr->K > (1 << 30)) return COMPASS_ERR_UNSUPPORTED;
+  return COMPASS_OK;
+}
+
+int validate_pointers(const void* const* a, const void* const* b, void* const* o, int P) {
+  if (a == nullptr || b == nullptr || o == nullptr) return COMPASS_ERR_INVALID_ARG;
+  for (int r = 0; r < P; ++r)
+    if (a[r] == nullptr || b[r] == nullptr || o[r] == nullptr) return COMPASS_ERR_INVALID_ARG;
+  for (int r = 0; r < P; ++r)
+    if (!aligned16(a[r]) || !aligned16(b[r]) || !aligned16(o[r])) return COMPASS_ERR_ALIGNMENT;
+  return COMPASS_OK;
+}
+
+int validate_workspace(const compass_problem* pr, int which, void* ws, size_t ws_bytes) {
+  size_t need = 0;
+  int st = compass_workspace_bytes(pr, which, &need);
+  if (st != COMPASS_OK) return st;
+  if (ws == nullptr) return COMPASS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0) return COMPASS_ERR_ALIGNMENT;
+  if (ws_bytes < need) return COMPASS_ERR_BUFFER_TOO_SMALL;
+  return COMPASS_OK;
+}
+
+inline int tiles_of(int64_t rows, int tile) { return int((rows + tile - 1) / tile); }
+
+// Number of ring-RMW tile counters of a fused GEMM+ReduceScatter launch.
+size_t rmw_counter_count(const compass_problem* pr) {
+  const int64_t h = pr->M / pr->P / pr->rings;
+  return size_t(pr->rings) * size_t(pr->P) * size_t(tiles_of(h, BM)) * size_t(tiles_of(pr->N, BN));
+}
+
+// ---- fused launches: schedule -> blocks -------------------------------------
+
+// AllGather+GEMM: one block per schedule entry, listed step-major, then ring,
+// then rank, so that for every rank the blocks appear in its schedule order.
+void plan_ag(const compass_problem* pr, const compass_sched_entry* table, GemmLaunch* L, compass_plan_block* view) {
+  const int P = pr->P, rings = pr->rings;
+  const int64_t m = pr->M / P;
+  L->n_a = L->n_b = L->n_out = P;
+  L->a_rows = m;
+  L->K = pr->K;
+  L->N = pr->N;
+  L->ldo = pr->N;
+  L->n_seg = 1;
+  L->rows_per_block = int(m / rings);
+  L->epilogue = EPI_STORE;
+  int n = 0;
+  for (int step = 0; step < P; ++step)
+    for (int ring = 0; ring < rings; ++ring)
+      for (int rank = 0; rank < P; ++rank) {
+        const compass_sched_entry& e = table[(size_t(rank) * P + step) * rings + ring];
+        BlockDesc& b = L->blocks[n];
+        std::memset(&b, 0, sizeof(b));
+        b.a_map = uint8_t(e.chunk);                       // read the owner's shard: gather by address
+        b.a_row0 = e.row_begin - e.chunk * int32_t(m);
+        b.b_map = uint8_t(rank);
+        b.out_idx = uint8_t(rank);
+        b.out_row0 = e.row_begin;
+        b.step = uint8_t(step);
+        b.part = uint8_t(e.part);
+        if (view) {
+          compass_plan_block& v = view[n];
+          v.rank = rank; v.step = step; v.ring = ring; v.part = e.part;
+          v.a_tensor = e.chunk; v.a_row_begin = b.a_row0;
+          v.out_tensor = rank; v.out_row_begin = b.out_row0;
+          v.rows = e.row_count;
+        }
+        ++n;
+      }
+  L->n_blocks = n;
+}
+
+// GEMM+ReduceScatter, segmented K: one block per partition; segment s of the
+// k-loop reads the rank that contributes at step s of the ring.
+void plan_rs_segmented(const compass_problem* pr, const compass_sched_entry* table, GemmLaunch* L,
+                       compass_plan_block* view) {
+  const int P = pr->P, rings = pr->rings;
+  const int64_t m = pr->M / P;
+  const int64_t h = m / rings;
+  L->n_a = L->n_b = L->n_out = P;
+  L->a_rows = pr->M;
+  L->K = pr->K;
+  L->N = pr->N;
+  L->ldo = pr->N;
+  L->n_seg = P;
+  L->rows_per_block = int(h);
+  L->epilogue = EPI_STORE;
+  const int n_parts = rings * P;
+  for (int part = 0; part < n_parts; ++part) {
+    const int chunk = part / rings, ring = part % rings;
+    BlockDesc& b = L->blocks[part];
+    std::memset(&b, 0, sizeof(b));
+    b.a_row0 = int32_t(chunk * m + ring * h);
+    b.out_idx = uint8_t(chunk);
+    b.out_row0 = int32_t(ring * h);
+    b.step = uint8_t(P - 1);
+    b.part = uint8_t(part);
+    if (view) {
+      compass_plan_block& v = view[part];
+      v.rank = -1; v.step = P - 1; v.ring = ring; v.part = part;
+      v.a_tensor = -1; v.a_row_begin = b.a_row0;
+      v.out_tensor = chunk; v.out_row_begin = b.out_row0;
+      v.rows = int32_t(h);
+    }
+  }
+  for (int rank = 0; rank < P; ++rank)
+    for (int step = 0; step < P; ++step)
+      for (int ring = 0; ring < rings; ++ring) {
+        const compass_sched_entry& e = table[(size_t(rank) * P + step) * rings + ring];
+        L->seg_rank[e.part][step] = uint8_t(rank);
+      }
+  L->n_blocks = n_parts;
+}
+
+// GEMM+ReduceScatter, ring read-modify-write: one block per schedule entry in
+// the same launch order as AllGather+GEMM; contributor `step` of a partition
+// precedes contributor step+1 in the launch.
+void plan_rs_ring(const compass_problem* pr, const compass_sched_entry* table, GemmLaunch* L, compass_plan_block* view) {
+  const int P = pr->P, rings = pr->rings;
+  const int64_t m = pr->M / P;
+  L->n_a = L->n_b = L->n_out = P;
+  L->a_rows = pr->M;
+  L->K = pr->K;
+  L->N = pr->N;
+  L->ldo = pr->N;
+  L->n_seg = 1;
+  L->rows_per_block = int(m / rings);
+  L->epilogue = EPI_RING_RMW;
+  L->last_step = P - 1;
+  int n = 0;
+  for (int step = 0; step < P; ++step)
+    for (int ring = 0; ring < rings; ++ring)
+      for (int rank = 0; rank < P; ++rank) {
+        const compass_sched_entry& e = table[(size_t(rank) * P + step) * rings + ring];
+        BlockDesc& b = L->blocks[n];
+        std::memset(&b, 0, sizeof(b));
+        b.a_map = uint8_t(rank);
+        b.b_map = uint8_t(rank);
+        b.a_row0 = e.row_begin;
+        b.out_idx = uint8_t(e.chunk);
+        b.out_row0 = e.row_begin - e.chunk * int32_t(m);
+        b.step = uint8_t(step);
+        b.part = uint8_t(e.part);
+        if (view) {
+          compass_plan_block& v = view[n];
+          v.rank = rank; v.step = step; v.ring = ring; v.part = e.part;
+          v.a_tensor = rank; v.a_row_begin = b.a_row0;
+          v.out_tensor = e.chunk; v.out_row_begin = b.out_row0;
+          v.rows = e.row_count;
+        }
+        ++n;
+      }
+  L->n_blocks = n;
+}
+
+int plan_fused(const compass_problem* pr, GemmLaunch* L, compass_plan_block* view) {
+  static thread_local compass_sched_entry table[kMaxBlocks];
+  int st = validate_schedule_args(pr->op, pr->P, pr->rings, pr->M);
+  if (st != COMPASS_OK) return st;
+  build_schedule(pr->op, pr->P, pr->rings, pr->M, table);
+  if (pr->op == COMPASS_OP_AG_GEMM) plan_ag(pr, table, L, view);
+  else if (pr->rs_variant == COMPASS_RS_SEGMENTED_K) plan_rs_segmented(pr, table, L, view);
+  else plan_rs_ring(pr, table, L, view);
+  if (view) {
+    const int per_block = tiles_of(L->rows_per_block, BM) * tiles_of(L->N, BN);
+    for (int i = 0; i < L->n_blocks; ++i) {
+      view[i].first_tile = i * per_block;
+      view[i].tile_count = per_block;
+    }
+  }
+  return COMPASS_OK;
+}
+
+int fused_call(const compass_problem* pr, int op, const void* const* A, const void* const* B, void* const* out, void* ws,
+               size_t ws_bytes, void* stream) {
+  int st = validate_problem(pr, op, false);
+  if (st != COMPASS_OK) return st;
+  st = validate_pointers(A, B, out, pr->P);
+  if (st != COMPASS_OK) return st;
+  st = validate_workspace(pr, COMPASS_WS_FUSED, ws, ws_bytes);
+  if (st != COMPASS_OK) return st;
+  if (op == COMPASS_OP_GEMM_RS && pr->rs_variant == COMPASS_RS_RING_RMW) return COMPASS_ERR_UNSUPPORTED;
+  static thread_local GemmLaunch L;
+  st = plan_fused(pr, &L, nullptr);
+  if (st != COMPASS_OK) return st;
+  for (int r = 0; r < pr->P; ++r) {
+    L.a_ptr[r] = A[r];
+    L.b_ptr[r] = B[r];
+    L.out_ptr[r] = out[r];
+  }
+  L.status = static_cast<StatusBlock*>(ws);
+  L.tile_counters = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + COMPASS_STATUS_BYTES);
+  return launch_gemm(L, static_cast<cudaStream_t>(stream));
+}
+
+// ---- InterDecom ----------------------------------------------------------------
+
+struct EventPool {
+  std::mutex mu;
+  cudaEvent_t ev[2 * 16 + 2];
+  int made = 0;
+  int ensure(int n) {
+    while (made < n) {
+      cudaError_t e = cudaEventCreateWithFlags(&ev[made], cudaEventDisableTiming);
+      if (e != cudaSuccess) return record_cuda_error(e);
+      ++made;
+    }
+    return COMPASS_OK;
+  }
+};
+EventPool g_events;
+
+int decomp_ag(const compass_problem* pr, const void* const* A, const void* const* B, void* const* C, uint8_t* ws,
+              cudaStream_t s_comp, cudaStream_t s_copy, cudaEvent_t* ev) {
+  const int P = pr->P, d = pr->d;
+  const int64_t m = pr->M / P, K = pr->K, sl = m / d;
+  const size_t gather_bytes = align_up(size_t(pr->M) * size_t(K) * 2);
+  uint8_t* G[kMaxP];
+  for (int r = 0; r < P; ++r) G[r] = ws + COMPASS_STATUS_BYTES + size_t(r) * gather_bytes;
+
+  static thread_local GemmLaunch L;
+  L.n_a = L.n_b = L.n_out = P;
+  L.a_rows = pr->M;
+  L.K = K;
+  L.N = pr->N;
+  L.ldo = pr->N;
+  L.n_seg = 1;
+  L.rows_per_block = int(sl);
+  L.epilogue = EPI_STORE;
+  L.status = reinterpret_cast<StatusBlock*>(ws);
+  L.tile_counters = nullptr;
+  for (int r = 0; r < P; ++r) {
+    L.a_ptr[r] = G[r];
+    L.b_ptr[r] = B[r];
+    L.out_ptr[r] = C[r];
+  }
+  cudaError_t e;
+  // the copy stream starts after whatever precedes this call on the compute stream
+  if ((e = cudaEventRecord(ev[0], s_comp)) != cudaSuccess) return record_cuda_error(e);
+  if ((e = cudaStreamWaitEvent(s_copy, ev[0], 0)) != cudaSuccess) return record_cuda_error(e);
+  for (int j = 0; j < d; ++j) {
+    // sub-AllGather j: row slice j of every shard into every rank's gather buffer
+    for (int r = 0; r < P; ++r)
+      for (int q = 0; q < P; ++q) {
+        const uint8_t* src = static_cast<const uint8_t*>(A[q]) + size_t(j * sl) * size_t(K) * 2;
+        uint8_t* dst = G[r] + size_t(q * m + j * sl) * size_t(K) * 2;
+        e = cudaMemcpyAsync(dst, src, size_t(sl) * size_t(K) * 2, cudaMemcpyDeviceToDevice, s_copy);
+        if (e != cudaSuccess) return record_cuda_error(e);
+      }
+    if ((e = cudaEventRecord(ev[1 + j], s_copy)) != cudaSuccess) return record_cuda_error(e);
+    if ((e = cudaStreamWaitEvent(s_comp, ev[1 + j], 0)) != cudaSuccess) return record_cuda_error(e);
+    // sub-GEMM j on the gathered rows
+    int n = 0;
+    for (int q = 0; q < P; ++q)
+      for (int r = 0; r < P; ++r) {
+        BlockDesc& b = L.blocks[n++];
+        std::memset(&b, 0, sizeof(b));
+        b.a_map = uint8_t(r);
+        b.b_map = uint8_t(r);
+        b.out_idx = uint8_t(r);
+        b.a_row0 = int32_t(q * m + j * sl);
+        b.out_row0 = b.a_row0;
+      }
+    L.n_blocks = n;
+    int st = launch_gemm(L, s_comp);
+    if (st != COMPASS_OK) return st;
+  }
+  return COMPASS_OK;
+}
+
+int decomp_rs(const compass_problem* pr, const void* const* A, const void* const* B, void* const* Out, uint8_t* ws,
+              cudaStream_t s_comp, cudaStream_t s_copy, cudaEvent_t* ev) {
+  const int P = pr->P, d = pr->d;
+  const int64_t m = pr->M / P, sl = m / d;
+  const size_t partial_bytes = align_up(size_t(pr->M) * size_t(pr->N) * 2);
+  void* W[kMaxP];
+  for (int q = 0; q < P; ++q) W[q] = ws + COMPASS_STATUS_BYTES + size_t(q) * partial_bytes;
+
+  static thread_local GemmLaunch L;
+  L.n_a = L.n_b = L.n_out = P;
+  L.a_rows = pr->M;
+  L.K = pr->K;
+  L.N = pr->N;
+  L.ldo = pr->N;
+  L.n_seg = 1;
+  L.rows_per_block = int(sl);
+  L.epilogue = EPI_STORE;
+  L.status = reinterpret_cast<StatusBlock*>(ws);
+  L.tile_counters = nullptr;
+  for (int q = 0; q < P; ++q) {
+    L.a_ptr[q] = A[q];
+    L.b_ptr[q] = B[q];
+    L.out_ptr[q] = W[q];
+  }
+  cudaError_t e;
+  for (int j = 0; j < d; ++j) {
+    // sub-GEMM j: every rank's partial rows of slice j of every owner's block
+    int n = 0;
+    for (int c = 0; c < P; ++c)
+      for (int q = 0; q < P; ++q) {
+        BlockDesc& b = L.blocks[n++];
+        std::memset(&b, 0, sizeof(b));
+        b.a_map = uint8_t(q);
+        b.b_map = uint8_t(q);
+        b.out_idx = uint8_t(q);
+        b.a_row0 = int32_t(c * m + j * sl);
+        b.out_row0 = b.a_row0;
+      }
+    L.n_blocks = n;
+    int st = launch_gemm(L, s_comp);
+    if (st != COMPASS_OK) return st;
+    if ((e = cudaEventRecord(ev[1 + j], s_comp)) != cudaSuccess) return record_cuda_error(e);
+    if ((e = cudaStreamWaitEvent(s_copy, ev[1 + j], 0)) != cudaSuccess) return record_cuda_error(e);
+    // sub-ReduceScatter j
+    st = launch_reduce_partials(W, P, Out, m, pr->N, j * sl, sl, s_copy);
+    if (st != COMPASS_OK) return st;
+  }
+  // later work on the compute stream sees the reduced output
+  if ((e = cudaEventRecord(ev[0], s_copy)) != cudaSuccess) return record_cuda_error(e);
+  if ((e = cudaStreamWaitEvent(s_comp, ev[0], 0)) != cudaSuccess) return record_cuda_error(e);
+  return COMPASS_OK;
+}
+
+}  // namespace
+
+int record_cuda_error(cudaError_t e) {
+  g_last_cuda_error.store(int(e));
+  return COMPASS_ERR_CUDA;
+}
+void count_kernel_launch() { g_kernel_launches.fetch_add(1, std::memory_order_relaxed); }
+
+}  // namespace compass
+
+using namespace compass;
+
+extern "C" int compass_workspace_bytes(const compass_problem* pr, int which, size_t* bytes) {
+  if (bytes == nullptr) return COMPASS_ERR_INVALID_ARG;
+  if (which != COMPASS_WS_FUSED && which != COMPASS_WS_DECOMP) return COMPASS_ERR_INVALID_ARG;
+  int st = validate_problem(pr, -1, which == COMPASS_WS_DECOMP);
+  if (st != COMPASS_OK) return st;
+  size_t total = COMPASS_STATUS_BYTES;
+  if (which == COMPASS_WS_FUSED) {
+    if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant == COMPASS_RS_RING_RMW)
+      total += align_up(rmw_counter_count(pr) * sizeof(int32_t));
+  } else {
+    const size_t inner = pr->op == COMPASS_OP_AG_GEMM ? size_t(pr->K) : size_t(pr->N);
+    total += size_t(pr->P) * align_up(size_t(pr->M) * inner * 2);
+  }
+  *bytes = total;
+  return COMPASS_OK;
+}
+
+extern "C" int compass_workspace_init(void* ws, size_t ws_bytes, void* stream) {
+  if (ws == nullptr || ws_bytes < COMPASS_STATUS_BYTES) return COMPASS_ERR_INVALID_ARG;
+  cudaError_t e = cudaMemsetAsync(ws, 0, ws_bytes, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return record_cuda_error(e);
+  return COMPASS_OK;
+}
+
+extern "C" int compass_read_status(void* ws, void* stream, int* detail) {
+  if (ws == nullptr) return COMPASS_ERR_INVALID_ARG;
+  StatusBlock host;
+  cudaError_t e = cudaMemcpyAsync(&host, ws, sizeof(host), cudaMemcpyDeviceToHost, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return record_cuda_error(e);
+  e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return record_cuda_error(e);
+  if (detail) *detail = host.detail;
+  return host.code;
+}
+
+extern "C" int compass_launch_plan(const compass_problem* pr, compass_plan_block* out, size_t capacity, size_t* count) {
+  if (count == nullptr) return COMPASS_ERR_INVALID_ARG;
+  int st = validate_problem(pr, -1, false);
+  if (st != COMPASS_OK) return st;
+  const bool per_entry = pr->op == COMPASS_OP_AG_GEMM || pr->rs_variant == COMPASS_RS_RING_RMW;
+  const size_t n = size_t(pr->rings) * pr->P * (per_entry ? pr->P : 1);
+  *count = n;
+  if (out == nullptr) return COMPASS_OK;
+  if (capacity < n) return COMPASS_ERR_BUFFER_TOO_SMALL;
+  static thread_local GemmLaunch L;
+  static thread_local compass_plan_block view[kMaxBlocks];
+  st = plan_fused(pr, &L, view);
+  if (st != COMPASS_OK) return st;
+  std::memcpy(out, view, n * sizeof(compass_plan_block));
+  return COMPASS_OK;
+}
+
+extern "C" int compass_ag_gemm(const compass_problem* pr, const void* const* A, const void* const* B, void* const* C,
+                               void* ws, size_t ws_bytes, void* stream) {
+  return fused_call(pr, COMPASS_OP_AG_GEMM, A, B, C, ws, ws_bytes, stream);
+}
+
+extern "C" int compass_gemm_rs(const compass_problem* pr, const void* const* A, const void* const* B, void* const* Out,
+                               void* ws, size_t ws_bytes, void* stream) {
+  return fused_call(pr, COMPASS_OP_GEMM_RS, A, B, Out, ws, ws_bytes, stream);
+}
+
+extern "C" int compass_decomp(const compass_problem* pr, const void* const* A, const void* const* B, void* const* out,
+                              void* ws, size_t ws_bytes, void* stream_compute, void* stream_copy) {
+  int st = validate_problem(pr, -1, true);
+  if (st != COMPASS_OK) return st;
+  if (pr->d > 16) return COMPASS_ERR_UNSUPPORTED;
+  st = validate_pointers(A, B, out, pr->P);
+  if (st != COMPASS_OK) return st;
+  st = validate_workspace(pr, COMPASS_WS_DECOMP, ws, ws_bytes);
+  if (st != COMPASS_OK) return st;
+  std::lock_guard<std::mutex> lock(g_events.mu);
+  st = g_events.ensure(pr->d + 1);
+  if (st != COMPASS_OK) return st;
+  cudaStream_t sc = static_cast<cudaStream_t>(stream_compute), sp = static_cast<cudaStream_t>(stream_copy);
+  if (pr->op == COMPASS_OP_AG_GEMM) return decomp_ag(pr, A, B, out, static_cast<uint8_t*>(ws), sc, sp, g_events.ev);
+  return decomp_rs(pr, A, B, out, static_cast<uint8_t*>(ws), sc, sp, g_events.ev);
+}
+
+extern "C" int compass_fused_host(const compass_problem* pr, const void* const* A_host, const void* const* B_host,
+                                  void* const* out_host, void* staging, size_t staging_bytes, size_t* needed, void* ws,
+                                  size_t ws_bytes, void* stream) {
+  int st = validate_problem(pr, -1, false);
+  if (st != COMPASS_OK) return st;
+  const int P = pr->P;
+  const bool ag = pr->op == COMPASS_OP_AG_GEMM;
+  const size_t a_bytes = size_t(ag ? pr->M / P : pr->M) * size_t(pr->K) * 2;
+  const size_t b_bytes = size_t(pr->N) * size_t(pr->K) * 2;
+  const size_t o_bytes = size_t(ag ? pr->M : pr->M / P) * size_t(pr->N) * 2;
+  const size_t total = size_t(P) * (align_up(a_bytes) + align_up(b_bytes) + align_up(o_bytes));
+  if (needed) *needed = total;
+  if (staging == nullptr) return needed ? COMPASS_OK : COMPASS_ERR_INVALID_ARG;
+  if (staging_bytes < total) return COMPASS_ERR_BUFFER_TOO_SMALL;
+  if ((reinterpret_cast<uintptr_t>(staging) & (kAlign - 1)) != 0) return COMPASS_ERR_ALIGNMENT;
+  if (A_host == nullptr || B_host == nullptr || out_host == nullptr) return COMPASS_ERR_INVALID_ARG;
+  for (int r = 0; r < P; ++r)
+    if (!A_host[r] || !B_host[r] || !out_host[r]) return COMPASS_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* base = static_cast<uint8_t*>(staging);
+  const void* dA[kMaxP];
+  const void* dB[kMaxP];
+  void* dO[kMaxP];
+  for (int r = 0; r < P; ++r) {
+    dA[r] = base + size_t(r) * align_up(a_bytes);
+    dB[r] = base + size_t(P) * align_up(a_bytes) + size_t(r) * align_up(b_bytes);
+    dO[r] = base + size_t(P) * (align_up(a_bytes) + align_up(b_bytes)) + size_t(r) * align_up(o_bytes);
+  }
+  cudaError_t e;
+  for (int r = 0; r < P; ++r) {
+    if ((e = cudaMemcpyAsync(const_cast<void*>(dA[r]), A_host[r], a_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+      return record_cuda_error(e);
+    if ((e = cudaMemcpyAsync(const_cast<void*>(dB[r]), B_host[r], b_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+      return record_cuda_error(e);
+  }
+  st = fused_call(pr, pr->op, dA, dB, dO, ws, ws_bytes, stream);
+  if (st != COMPASS_OK) return st;
+  for (int r = 0; r < P; ++r)
+    if ((e = cudaMemcpyAsync(out_host[r], dO[r], o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
+      return record_cuda_error(e);
+  return COMPASS_OK;
+}
+
+extern "C" const char* compass_status_string(int status) {
+  switch (status) {
+    case COMPASS_OK: return "ok";
+    case COMPASS_ERR_INVALID_ARG: return "invalid argument";
+    case COMPASS_ERR_SHAPE: return "shape not divisible as required";
+    case COMPASS_ERR_UNSUPPORTED: return "unsupported dtype or size";
+    case COMPASS_ERR_ALIGNMENT: return "pointer or row pitch not 16-byte aligned";
+    case COMPASS_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+    case COMPASS_ERR_CUDA: return "CUDA call failed";
+    case COMPASS_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int compass_last_cuda_error(void) { return g_last_cuda_error.load(); }
+extern "C" uint64_t compass_kernel_launch_count(void) { return g_kernel_launches.load(); }

@@ -1,0 +1,85 @@
+// HBM-bound helper kernels of the InterDecom path (Section II-B): the
+// sub-ReduceScatter that sums the P ranks' BF16 partial rows of one row slice
+// into the owners' output rows (FP32 accumulation, ranks in ascending order,
+// one BF16 rounding).
+#include "internal.h"
+#include "ptx_sm100.cuh"
+
+namespace compass {
+
+namespace {
+
+struct ReduceParams {
+  const uint4* partial[kMaxP];   // [M x N] BF16 each
+  uint4* out[kMaxP];             // [m x N] BF16 each
+  int32_t P;
+  int64_t m;                     // rows per owner
+  int64_t n_vec;                 // N / 8 (16-byte vectors per row)
+  int64_t slice_begin;           // first row of the slice inside every owner's block
+  int64_t slice_rows;
+};
+
+__device__ __forceinline__ void accumulate_bf16x8(float (&acc)[8], const uint4& v) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    acc[2 * i + 0] += __uint_as_float(w[i] << 16);
+    acc[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
+__global__ void __launch_bounds__(256) reduce_partials_kernel(const __grid_constant__ ReduceParams p) {
+  const int64_t per_owner = p.slice_rows * p.n_vec;
+  const int64_t total = per_owner * p.P;
+  for (int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += int64_t(gridDim.x) * blockDim.x) {
+    const int c = int(i / per_owner);
+    const int64_t w = i - int64_t(c) * per_owner;
+    const int64_t row = w / p.n_vec;
+    const int64_t col = w - row * p.n_vec;
+    const int64_t src = (int64_t(c) * p.m + p.slice_begin + row) * p.n_vec + col;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int q = 0; q < p.P; ++q) accumulate_bf16x8(acc, __ldg(p.partial[q] + src));
+    uint4 r;
+    r.x = ptx::pack_bf16x2(acc[0], acc[1]);
+    r.y = ptx::pack_bf16x2(acc[2], acc[3]);
+    r.z = ptx::pack_bf16x2(acc[4], acc[5]);
+    r.w = ptx::pack_bf16x2(acc[6], acc[7]);
+    p.out[c][(p.slice_begin + row) * p.n_vec + col] = r;
+  }
+}
+
+}  // namespace
+
+int launch_reduce_partials(const void* const* partial, int P, void* const* out, int64_t m, int64_t N, int64_t slice_begin,
+                           int64_t slice_rows, cudaStream_t stream) {
+  ReduceParams p;
+  for (int q = 0; q < P; ++q) {
+    p.partial[q] = static_cast<const uint4*>(partial[q]);
+    p.out[q] = static_cast<uint4*>(out[q]);
+  }
+  p.P = P;
+  p.m = m;
+  p.n_vec = N / 8;
+  p.slice_begin = slice_begin;
+  p.slice_rows = slice_rows;
+  const int64_t total = slice_rows * p.n_vec * P;
+  if (total <= 0) return COMPASS_OK;
+  static int num_sms = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+  }
+  int64_t want = (total + 255) / 256;
+  int64_t cap = int64_t(num_sms) * 8;
+  int grid = int(want < cap ? want : cap);
+  reduce_partials_kernel<<<grid, 256, 0, stream>>>(p);
+  count_kernel_launch();
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return record_cuda_error(e);
+  return COMPASS_OK;
+}
+
+}  // namespace compass

@@ -1,0 +1,119 @@
+// Structures shared between the host-side planner and the kernels.
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/compass.h"
+
+namespace compass {
+
+constexpr int kMaxP = COMPASS_MAX_P;
+constexpr int kMaxBlocks = 2 * kMaxP * kMaxP;   // rings * P * P schedule entries
+constexpr int kMaxSegBlocks = 2 * kMaxP;        // blocks of a segmented-K launch (rings * P partitions)
+
+// Tile shape of the GEMM kernel (one CTA computes BM x BN of the output).
+constexpr int BM = 128;
+constexpr int BN = 256;
+constexpr int BK = 64;          // 64 BF16 = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;
+
+// Device status block at the start of a workspace.
+struct StatusBlock {
+  int32_t code;      // compass_status
+  int32_t detail;    // which wait gave up (WaitSite) and where
+  int32_t block_idx;
+  int32_t tile;
+};
+
+enum WaitSite : int32_t {
+  WAIT_NONE = 0,
+  WAIT_SMEM_EMPTY = 1,     // TMA producer waiting for a free pipeline stage
+  WAIT_SMEM_FULL = 2,      // MMA issuer waiting for operands
+  WAIT_ACC_EMPTY = 3,      // MMA issuer waiting for a free accumulator
+  WAIT_ACC_FULL = 4,       // epilogue waiting for an accumulator
+  WAIT_DRAIN = 5,          // teardown waiting for outstanding work
+  WAIT_TILE_COUNTER = 6,   // ring read-modify-write waiting for the previous contributor
+};
+
+// A block is a contiguous range of output rows handled as tiles_m x tiles_n
+// tiles.  For the fused kernels one block = one schedule entry.
+struct BlockDesc {
+  int32_t a_row0;     // first row read from the A tensor(s)
+  int32_t out_row0;   // first row written in the output tensor
+  uint8_t a_map;      // index of the A tensor map (single-segment launches)
+  uint8_t b_map;      // index of the B tensor map (single-segment launches)
+  uint8_t out_idx;    // index of the output pointer
+  uint8_t step;       // schedule step (ring read-modify-write: contributor index)
+  uint8_t part;       // schedule partition id
+  uint8_t pad[3];
+};
+
+enum EpilogueMode : int32_t {
+  EPI_STORE = 0,      // round to BF16 and store
+  EPI_RING_RMW = 1,   // ordered accumulate into the output in ring order
+};
+
+struct GemmParams {
+  CUtensorMap a_maps[kMaxP];
+  CUtensorMap b_maps[kMaxP];
+  __nv_bfloat16* out[kMaxP];
+  int64_t ldo;             // output row pitch in elements
+  int32_t n_blocks;
+  int32_t rows_per_block;
+  int32_t N;               // output columns
+  int32_t n_seg;           // K segments accumulated into one tile (1, or P for segmented-K reduce)
+  int32_t kb_per_seg;      // k-blocks of BK per segment (last one may be partial)
+  int32_t tail_ksteps;     // UMMA_K steps in the last k-block of a segment (1..BK/UMMA_K)
+  int32_t tiles_m, tiles_n;
+  int32_t total_tiles;
+  int32_t epilogue;        // EpilogueMode
+  int32_t last_step;       // ring RMW: step index of the final contributor (P-1)
+  uint32_t wait_limit_us;  // bound of every device-side wait
+  StatusBlock* status;
+  int32_t* tile_counters;  // ring RMW only
+  uint8_t seg_rank[kMaxSegBlocks][kMaxP];   // segmented-K: tensor index of segment s of block b
+  BlockDesc blocks[kMaxBlocks];
+};
+
+// Host-side description of a GEMM launch before tensor maps are encoded.
+struct GemmLaunch {
+  const void* a_ptr[kMaxP];
+  const void* b_ptr[kMaxP];
+  void* out_ptr[kMaxP];
+  int n_a = 0, n_b = 0, n_out = 0;
+  int64_t a_rows = 0;      // rows of every A tensor
+  int64_t K = 0;           // columns (contraction length) of every A and B tensor
+  int64_t N = 0;           // rows of every B tensor = output columns
+  int64_t ldo = 0;
+  int n_seg = 1;
+  int rows_per_block = 0;
+  int epilogue = EPI_STORE;
+  int last_step = 0;
+  int n_blocks = 0;
+  BlockDesc blocks[kMaxBlocks];
+  uint8_t seg_rank[kMaxSegBlocks][kMaxP];
+  StatusBlock* status = nullptr;
+  int32_t* tile_counters = nullptr;
+};
+
+// gemm_sm100.cu
+int launch_gemm(const GemmLaunch& launch, cudaStream_t stream);
+size_t gemm_smem_bytes();
+
+// aux_kernels.cu
+int launch_reduce_partials(const void* const* partial, int P, void* const* out, int64_t m, int64_t N,
+                           int64_t slice_begin, int64_t slice_rows, cudaStream_t stream);
+
+// api.cu
+int record_cuda_error(cudaError_t e);
+void count_kernel_launch();
+
+// schedule.cpp
+int build_schedule(int op, int P, int rings, int64_t M, compass_sched_entry* out);   // out has rings*P*P slots
+int validate_schedule_args(int op, int P, int rings, int64_t M);
+
+}  // namespace compass

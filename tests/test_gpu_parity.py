@@ -1,0 +1,201 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle
+on the same seeded inputs.
+
+Acceptance (every element of every rank's output):
+    |gpu - ref| <= 1e-2 * max|ref| + 1e-3         (BF16 output, FP32 accumulate)
+plus RMS error <= 2^-8 of the reference RMS (oracle.compare).  Schedules are
+compared bit-exactly.  Small cases are checked element by element; the
+full-size configurations on a row sample (rows next to every partition and
+tile boundary plus 1 % random rows, full width)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import compare
+from oracle import operators as ops
+from oracle.schedule import schedule as oracle_schedule
+from paper_2609_10549_b200 import api
+from paper_2609_10549_b200 import workloads as wl
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+def check_all(outs, refs, what):
+    for r, (got, ref) in enumerate(zip(outs, refs)):
+        rep = compare.check(got, ref)
+        assert rep.ok, f"{what} rank {r}: {rep}"
+
+
+def small(op, P, m, N, K, seed=1, dist=1.0):
+    return wl.Workload(f"small-{op}-{P}-{m}-{N}-{K}", op, P=P, M=P * m, N=N, K=K,
+                       a_dist=("normal", 1.0), b_dist=("normal", dist), seed=seed)
+
+
+def test_library_was_loaded_and_counts_launches():
+    before = api.kernel_launch_count()
+    w = small(wl.OP_AG_GEMM, 1, 128, 256, 64)
+    A, B = wl.make_inputs(w)
+    outs, status, guards = gu.run_fused(w, A, B)
+    assert status == (api.OK, 0) and guards
+    assert api.kernel_launch_count() == before + 1
+    check_all(outs, ops.ag_gemm(A, B), w.name)
+
+
+def test_config1_ag_gemm_full():
+    w = wl.C1_AG
+    A, B = wl.make_inputs(w)
+    assert np.array_equal(api.compass_schedule(w.op, w.P, 2, w.M), oracle_schedule(w.op, w.P, 2, w.M))
+    outs, status, guards = gu.run_fused(w, A, B)
+    assert status == (api.OK, 0) and guards
+    check_all(outs, ops.ag_gemm(A, B), w.name)
+
+
+# (P, rows per rank, N, K, rings): several tiles, ragged tails in M, N and K,
+# partitions smaller than a tile, K shorter than one k-block, odd P.
+AG_SHAPES = [
+    (1, 128, 256, 64, 2), (1, 256, 512, 128, 1), (2, 256, 256, 256, 2), (2, 144, 264, 72, 2),
+    (3, 272, 520, 1376, 2), (4, 512, 768, 512, 2), (4, 384, 1024, 320, 1), (8, 80, 200, 8, 2),
+    (5, 6, 8, 16, 2), (8, 256, 512, 192, 2), (16, 32, 64, 64, 2),
+]
+
+
+@pytest.mark.parametrize("P,m,N,K,rings", AG_SHAPES)
+def test_ag_gemm_small_shapes(P, m, N, K, rings):
+    w = small(wl.OP_AG_GEMM, P, m, N, K)
+    A, B = wl.make_inputs(w)
+    outs, status, guards = gu.run_fused(w, A, B, rings=rings)
+    assert status == (api.OK, 0) and guards
+    check_all(outs, ops.ag_gemm(A, B, rings=rings), w.name)
+
+
+RS_SHAPES = [
+    (1, 128, 256, 64, 2), (2, 256, 256, 256, 2), (2, 144, 264, 72, 2), (3, 272, 520, 344, 2),
+    (4, 512, 768, 512, 2), (4, 384, 1024, 320, 1), (8, 80, 200, 8, 2), (8, 256, 512, 1376, 2), (5, 6, 8, 16, 2),
+]
+
+
+@pytest.mark.parametrize("P,m,N,K,rings", RS_SHAPES)
+def test_gemm_rs_small_shapes(P, m, N, K, rings):
+    w = small(wl.OP_GEMM_RS, P, m, N, K, dist=0.05)
+    A, B = wl.make_inputs(w)
+    outs, status, guards = gu.run_fused(w, A, B, rings=rings)
+    assert status == (api.OK, 0) and guards
+    check_all(outs, ops.gemm_rs(A, B, rings=rings), w.name)
+
+
+@pytest.mark.parametrize("op", [wl.OP_AG_GEMM, wl.OP_GEMM_RS])
+def test_integer_inputs_are_reproduced_exactly(op):
+    """Small-integer inputs make every partial sum exact in FP32 and every
+    result exactly representable in BF16 after at most one rounding, so a
+    misplaced tile, row or k-slice shows up as an exact mismatch."""
+    w = wl.Workload("ints", op, P=4, M=4 * 256, N=512, K=192)
+    A, B = wl.make_structured_inputs(w, "index")
+    outs, status, guards = gu.run_fused(w, A, B)
+    assert status == (api.OK, 0) and guards
+    refs = ops.ag_gemm(A, B) if op == wl.OP_AG_GEMM else ops.gemm_rs(A, B)
+    for got, ref in zip(outs, refs):
+        assert np.array_equal(ops.bf16_bits_to_f64(got), ops.f64_to_bf16_f64(ref))
+
+
+def _sampled_ag(w, rings=2):
+    A, B = wl.make_inputs(w)
+    outs, status, guards = gu.run_fused(w, A, B, rings=rings)
+    assert status == (api.OK, 0) and guards
+    rows = gu.sample_rows(w.M, w.P, rings)
+    refs = ops.ag_gemm(A, B, rings=rings, rows=rows)
+    for r in range(w.P):
+        assert not np.any((outs[r] & 0x7F80) == 0x7F80), "NaN/Inf or unwritten output"
+        rep = compare.check(outs[r][rows], refs[r])
+        assert rep.ok, f"{w.name} rank {r}: {rep}"
+
+
+def _sampled_rs(w, rings=2, rs_variant=api.RS_SEGMENTED_K):
+    A, B = wl.make_inputs(w)
+    outs, status, guards = gu.run_fused(w, A, B, rings=rings, rs_variant=rs_variant)
+    assert status == (api.OK, 0) and guards
+    rows = gu.sample_rows(w.M, w.P, rings)
+    found = ops.gemm_rs_rows(A, B, rows, rings=rings)
+    assert sorted(found) == list(range(w.P))
+    for c, (local, ref) in found.items():
+        assert not np.any((outs[c] & 0x7F80) == 0x7F80), "NaN/Inf or unwritten output"
+        rep = compare.check(outs[c][local], ref)
+        assert rep.ok, f"{w.name} chunk {c}: {rep}"
+
+
+def test_config2_ag_gemm_full_size_sampled():
+    _sampled_ag(wl.C2_AG)
+
+
+def test_config3_gemm_rs_full_size_sampled():
+    _sampled_rs(wl.C3_RS)
+
+
+def test_config4_gemm_rs_full_size_sampled():
+    _sampled_rs(wl.C4_RS)
+
+
+def test_config5_ag_gemm_full_size_sampled():
+    _sampled_ag(wl.C5_AG)
+
+
+def test_config5_gemm_rs_full_size_sampled():
+    _sampled_rs(wl.C5_RS)
+
+
+@pytest.mark.parametrize("op,P,m,N,K,d", [
+    (wl.OP_AG_GEMM, 2, 256, 256, 128, 1), (wl.OP_AG_GEMM, 2, 256, 256, 128, 2), (wl.OP_AG_GEMM, 4, 512, 520, 200, 4),
+    (wl.OP_AG_GEMM, 4, 512, 256, 64, 16), (wl.OP_AG_GEMM, 3, 48, 64, 64, 8),
+    (wl.OP_GEMM_RS, 2, 256, 256, 128, 1), (wl.OP_GEMM_RS, 2, 256, 256, 128, 2), (wl.OP_GEMM_RS, 4, 512, 520, 200, 4),
+    (wl.OP_GEMM_RS, 4, 512, 256, 64, 16), (wl.OP_GEMM_RS, 3, 48, 64, 64, 8),
+])
+def test_interdecom_small_shapes(op, P, m, N, K, d):
+    w = small(op, P, m, N, K, dist=0.1)
+    A, B = wl.make_inputs(w)
+    outs, status, guards = gu.run_decomp(w, A, B, d)
+    assert status == (api.OK, 0) and guards
+    refs = ops.decomp_ag_gemm(A, B, d) if op == wl.OP_AG_GEMM else ops.decomp_gemm_rs(A, B, d)
+    check_all(outs, refs, f"{w.name} d={d}")
+
+
+@pytest.mark.parametrize("d", [1, 4, 16])
+def test_config4_interdecom_full_size_sampled(d):
+    for w in (wl.C4_AG, wl.C4_RS):
+        A, B = wl.make_inputs(w)
+        outs, status, guards = gu.run_decomp(w, A, B, d)
+        assert status == (api.OK, 0) and guards
+        rows = gu.sample_rows(w.M, w.P, 2, tile=max(1, w.m // d))
+        if w.op == wl.OP_AG_GEMM:
+            refs = ops.ag_gemm(A, B, rows=rows)
+            for r in range(w.P):
+                rep = compare.check(outs[r][rows], refs[r])
+                assert rep.ok, f"{w.name} d={d} rank {r}: {rep}"
+        else:
+            for c, (local, ref) in ops.gemm_rs_rows(A, B, rows).items():
+                rep = compare.check(outs[c][local], ref)
+                assert rep.ok, f"{w.name} d={d} chunk {c}: {rep}"
+
+
+@pytest.mark.parametrize("op", [wl.OP_AG_GEMM, wl.OP_GEMM_RS])
+def test_host_buffer_entry_point(op):
+    w = small(op, 2, 256, 264, 200, dist=0.1)
+    A, B = wl.make_inputs(w)
+    pr = gu.problem_of(w)
+    hA = [torch.from_numpy(a.view(np.int16)).pin_memory() for a in A]
+    hB = [torch.from_numpy(b.view(np.int16)).pin_memory() for b in B]
+    hO = [torch.full(w.out_shape, gu.NAN_BITS, dtype=torch.int16).pin_memory() for _ in range(w.P)]
+    staging = torch.empty(api.compass_fused_host_bytes(pr), dtype=torch.uint8, device="cuda")
+    ws = api.alloc_workspace(pr)
+    api.compass_fused_host(pr, hA, hB, hO, staging, ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    refs = ops.ag_gemm(A, B) if op == wl.OP_AG_GEMM else ops.gemm_rs(A, B)
+    check_all([o.numpy().view(np.uint16) for o in hO], refs, w.name)
+
+
+def test_repeated_calls_give_identical_bits():
+    w = small(wl.OP_GEMM_RS, 4, 512, 768, 512, dist=0.05)
+    A, B = wl.make_inputs(w)
+    first, _, _ = gu.run_fused(w, A, B)
+    second, _, _ = gu.run_fused(w, A, B)
+    for x, y in zip(first, second):
+        assert np.array_equal(x, y)

@@ -188,3 +188,15 @@ def test_acceptance_rule():
     drift = ref * 1.01
     rep = compare.check(wl.f32_to_bf16_bits(drift.astype(np.float32)), ref)
     assert rep.violations == 0 and not rep.ok
+
+
+def test_sampled_reduce_scatter_rows_equal_full_rows():
+    w, A, B = tiny(OP_GEMM_RS, 4, 64, 8, 16)
+    full = ops.gemm_rs(A, B)
+    rows = np.array([0, 7, 8, 15, 16, 40, 63])
+    got = ops.gemm_rs_rows(A, B, rows)
+    seen = 0
+    for c, (local, vals) in got.items():
+        assert np.array_equal(vals, full[c][local])
+        seen += len(local)
+    assert seen == len(rows)
