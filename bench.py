@@ -1,0 +1,386 @@
+"""Benchmark of the fused AllGather+GEMM / GEMM+ReduceScatter hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole hot path on the 7B-class layer pair: the ring
+schedule (host), the strategy selector (host), the fused AllGather+GEMM of the
+QKV projection (P=4, M=4096, K=4096, N=3072 per rank) and the fused
+GEMM+ReduceScatter of the MLP down projection (P=8, M=8192, K=1376 per rank,
+N=4096), on seeded synthetic BF16 data.  The metric is TFLOP/s over the FLOPs
+all logical ranks execute.  With N > 1 (torchrun) every rank runs an
+independent replica on its own GPU (the emulated tensor-parallel group lives
+on one GPU; there is no data-path collective) and the value is the aggregate.
+
+Prints ONE JSON line on rank 0.  `--impl reference` times the CPU oracle on a
+bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_10549_b200 import workloads as wl  # noqa: E402
+
+METRIC = "fused AG-GEMM + GEMM-RS throughput (7B-class layer pair)"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes per launch of the GEMM kernel from the ncu capture summarised in
+# profiles/ (null until a capture exists): {"C2": bytes, "C3": bytes}.
+NCU_TRAFFIC_BYTES = None
+
+
+def env_int(name, default):
+    try:
+        return int(os.environ.get(name, default))
+    except ValueError:
+        return default
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained")}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read only) while the
+    timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.005):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _loop(self):
+        nv = self._nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------------
+# the oracle on the host (reference arm and cpu_baseline leg)
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return int(max(n)) if n else 1
+    except Exception:
+        return 1
+
+
+class OracleSample:
+    """A bounded sample of the step for the CPU oracle: `rows_ag` rows of the
+    gathered activation for rank 0 of the AllGather+GEMM, and `rows_rs` rows of
+    the reduced tensor (all P contributions) of the GEMM+ReduceScatter."""
+
+    def __init__(self, w_ag, w_rs):
+        from oracle import operators as ops
+        self.ops = ops
+        self.w_ag, self.w_rs = w_ag, w_rs
+        self.A_ag, self.B_ag = wl.make_inputs(w_ag)
+        self.A_rs, self.B_rs = wl.make_inputs(w_rs)
+
+    def flops(self, rows_ag, rows_rs):
+        return 2.0 * rows_ag * self.w_ag.N * self.w_ag.K + 2.0 * rows_rs * self.w_rs.N * self.w_rs.K * self.w_rs.P
+
+    def run(self, rows_ag, rows_rs):
+        ra = np.linspace(0, self.w_ag.M - 1, rows_ag).astype(np.int64)
+        rr = np.unique(np.linspace(0, self.w_rs.M - 1, rows_rs).astype(np.int64))
+        self.ops.ag_gemm(self.A_ag, self.B_ag, ranks=[0], rows=ra)
+        self.ops.gemm_rs_rows(self.A_rs, self.B_rs, rr)
+
+    def size_for(self, seconds):
+        """Rows per operator so that one run takes about `seconds`."""
+        probe = (256, 128)
+        self.run(*probe)
+        t0 = time.perf_counter()
+        self.run(*probe)
+        dt = max(time.perf_counter() - t0, 1e-4)
+        scale = seconds / dt
+        ra = int(min(self.w_ag.M, max(64, probe[0] * scale)))
+        rr = int(min(self.w_rs.M, max(32, probe[1] * scale)))
+        return ra, rr
+
+
+def cpu_baseline(w_ag, w_rs, seconds=12.0):
+    s = OracleSample(w_ag, w_rs)
+    ra, rr = s.size_for(seconds)
+    t0 = time.perf_counter()
+    s.run(ra, rr)
+    dt = time.perf_counter() - t0
+    return {"value": s.flops(ra, rr) / dt / 1e12, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"{ra} of {w_ag.M} gathered rows of rank 0 ({w_ag.name}) + {rr} of {w_rs.M} reduced rows "
+                      f"with all {w_rs.P} contributions ({w_rs.name}), one pass, {dt:.1f} s, numpy FP64"}
+
+
+def run_reference(args, w_ag, w_rs):
+    rank = env_int("RANK", 0)
+    if rank != 0:
+        return
+    s = OracleSample(w_ag, w_rs)
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    ra, rr = s.size_for(min(budget, 10.0))
+    for _ in range(args.warmup):
+        s.run(ra, rr)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        s.run(ra, rr)
+    dt = time.perf_counter() - t0
+    value = s.flops(ra, rr) * args.steps / dt / 1e12
+    sample = (f"{ra} of {w_ag.M} gathered rows of rank 0 ({w_ag.name}) + {rr} of {w_rs.M} reduced rows with all "
+              f"{w_rs.P} contributions ({w_rs.name}) per step")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w_ag, w_rs),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w_ag, w_rs):
+    return {"workload": f"{w_ag.name} (P={w_ag.P}, M={w_ag.M}, K={w_ag.K}, N={w_ag.N}/rank) + "
+                        f"{w_rs.name} (P={w_rs.P}, M={w_rs.M}, K={w_rs.K}/rank, N={w_rs.N})",
+            "emulated_ranks": "P logical ranks on one GPU, separate HBM allocations per shard",
+            "l2": "inputs larger than L2: the two operators touch "
+                  f"{(w_ag.algorithmic_bytes + w_rs.algorithmic_bytes) / 1e6:.0f} MB per step (L2 = 126 MB)",
+            "multi_gpu": "replicas only"}
+
+
+# ---------------------------------------------------------------------------------
+# our arm
+
+def run_ours(args, w_ag, w_rs):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_10549_b200 import api
+    from paper_2609_10549_b200 import build as _build
+
+    rank, world, local = env_int("RANK", 0), env_int("WORLD_SIZE", 1), env_int("LOCAL_RANK", 0)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if rank == 0 or world == 1:
+        _build.build()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    api.lib()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    stream = torch.cuda.current_stream()
+
+    class Op:
+        def __init__(self, w):
+            self.w = w
+            self.pr = api.make_problem(w.op, w.P, w.M, w.N, w.K)
+            self.A_bits, self.B_bits = wl.make_inputs(w)
+            self.A = [api.to_device(a) for a in self.A_bits]
+            self.B = [api.to_device(b) for b in self.B_bits]
+            self.out = [torch.empty(w.out_shape, dtype=torch.bfloat16, device="cuda") for _ in range(w.P)]
+            self.ws = api.alloc_workspace(self.pr)
+            self.call = api.compass_ag_gemm if w.op == wl.OP_AG_GEMM else api.compass_gemm_rs
+
+        def run(self):
+            self.call(self.pr, self.A, self.B, self.out, self.ws, stream)
+
+    ag, rs = Op(w_ag), Op(w_rs)
+    calib = api.Calib(0.0, 1.0 / 1.2e15, 0.0, 1.0 / 3.0e12, 1.0, 0.02, 2e-6, 0.0)   # replaced by the sweep's fit below
+
+    def step(ev=None):
+        api.compass_schedule(w_ag.op, w_ag.P, 2, w_ag.M)
+        api.compass_schedule(w_rs.op, w_rs.P, 2, w_rs.M)
+        api.compass_select(ag.pr, calib)
+        api.compass_select(rs.pr, calib)
+        if ev is not None:
+            ev[0].record(stream)
+        ag.run()
+        if ev is not None:
+            ev[1].record(stream)
+        rs.run()
+        if ev is not None:
+            ev[2].record(stream)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    launches0 = api.kernel_launch_count()
+    with ClockSampler(local) as clocks:
+        t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        t_start.record(stream)
+        for i in range(args.steps):
+            step(events[i])
+        t_end.record(stream)
+        barrier()
+    launches = api.kernel_launch_count() - launches0
+    total_ms = t_start.elapsed_time(t_end)
+    status = (api.compass_read_status(ag.ws), api.compass_read_status(rs.ws))
+    if status != ((api.OK, 0), (api.OK, 0)):
+        raise SystemExit(f"device-side status after the timed region: {status}")
+    t_ag = float(np.mean([e[0].elapsed_time(e[1]) for e in events]))
+    t_rs = float(np.mean([e[1].elapsed_time(e[2]) for e in events]))
+
+    # end to end through the host-buffer entry point: pinned host inputs, H2D and D2H inside the timed region
+    e2e_steps = max(3, min(args.steps, 10))
+
+    class HostOp:
+        def __init__(self, op):
+            w = op.w
+            self.op = op
+            self.hA = [torch.from_numpy(a.view(np.int16)).pin_memory() for a in op.A_bits]
+            self.hB = [torch.from_numpy(b.view(np.int16)).pin_memory() for b in op.B_bits]
+            self.hO = [torch.empty(w.out_shape, dtype=torch.int16).pin_memory() for _ in range(w.P)]
+            self.staging = torch.empty(api.compass_fused_host_bytes(op.pr), dtype=torch.uint8, device="cuda")
+            self.h2d = sum(t.numel() * 2 for t in self.hA + self.hB)
+            self.d2h = sum(t.numel() * 2 for t in self.hO)
+
+        def run(self):
+            api.compass_fused_host(self.op.pr, self.hA, self.hB, self.hO, self.staging, self.op.ws, stream)
+
+    hag, hrs = HostOp(ag), HostOp(rs)
+    for _ in range(2):
+        hag.run(); hrs.run()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        api.compass_schedule(w_ag.op, w_ag.P, 2, w_ag.M)
+        api.compass_schedule(w_rs.op, w_rs.P, 2, w_rs.M)
+        api.compass_select(ag.pr, calib)
+        api.compass_select(rs.pr, calib)
+        hag.run(); hrs.run()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    # max over ranks
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_ms, t_ag, t_rs], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms, t_ag, t_rs = [float(x) for x in t.tolist()]
+        lt = torch.tensor([launches], dtype=torch.int64, device="cuda")
+        dist.all_reduce(lt, op=dist.ReduceOp.SUM)
+        launches = int(lt.item())
+
+    if rank == 0:
+        flops_step = w_ag.flops + w_rs.flops
+        ms_per_step = total_ms / args.steps
+        value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+        peaks, peak_src = measured_peaks()
+        kernel_s = (t_ag + t_rs) * 1e-3 / 2.0            # average duration of one launch of the GEMM kernel
+        achieved = (flops_step / 2.0) / kernel_s / 1e12
+        sustained = total_ms >= 1000.0
+        peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+        traffic = None
+        if NCU_TRAFFIC_BYTES:
+            traffic = (NCU_TRAFFIC_BYTES["C2"] + NCU_TRAFFIC_BYTES["C3"]) / 2.0
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(w_ag, w_rs),
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                         "frac": achieved / peak, "traffic": traffic,
+                         "peak_source": f"{'sustained' if sustained else 'burst'} cuBLAS bf16, of {peak_src}",
+                         "kernel": "gemm_kernel (two launches per step: AG-GEMM and GEMM-RS)",
+                         "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS},
+            "ag_gemm": {"ms": t_ag, "tflops": w_ag.flops / (t_ag * 1e-3) / 1e12,
+                        "frac_of_nominal_2250": w_ag.flops / (t_ag * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS},
+            "gemm_rs": {"ms": t_rs, "tflops": w_rs.flops / (t_rs * 1e-3) / 1e12,
+                        "frac_of_nominal_2250": w_rs.flops / (t_rs * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS},
+            "e2e": {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+                    "h2d_bytes_per_step": hag.h2d + hrs.h2d, "d2h_bytes_per_step": hag.d2h + hrs.d2h,
+                    "ms_per_step": e2e_ms, "steps": e2e_steps},
+            "gpu_launches": launches, "clocks": clocks.summary(),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(w_ag, w_rs)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w_ag, w_rs = wl.C2_AG, wl.C3_RS
+    if args.impl == "reference":
+        run_reference(args, w_ag, w_rs)
+    else:
+        run_ours(args, w_ag, w_rs)
+
+
+if __name__ == "__main__":
+    main()
