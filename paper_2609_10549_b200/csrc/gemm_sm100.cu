@@ -2,22 +2,30 @@
 //
 // One launch executes a list of "blocks" (contiguous output row ranges, for the
 // fused operators one block = one entry of the ring chunk schedule, Section
-// III-B) as 128x256 tiles.  Tile t of the launch is handled by CTA
-// (t mod gridDim.x); because the blocks are listed in schedule order, tiles are
-// issued to the SMs in schedule order.
+// III-B).  Tile t of the launch is handled by work unit (t mod #units);
+// because the blocks are listed in schedule order, tiles are issued to the SMs
+// in schedule order.
 //
 //   AllGather+GEMM: the A tile of a block is TMA-loaded straight from the shard
 //     of the rank that owns the partition (gather by address);
 //   GEMM+ReduceScatter, segmented K: the k-loop of a tile runs over the P ranks'
-//     K slices in ring order into one TMEM accumulator (in-kernel reduction);
-//   GEMM+ReduceScatter, ring RMW: the epilogue adds the partial tile into the
-//     owner's rows in ring order (ordered read-modify-write).
+//     K slices in ring order into one TMEM accumulator (in-kernel reduction).
+//
+// Two modes of the same kernel:
+//   pair   (default when a block has >= 256 rows): a cluster of two CTAs owns a
+//          256x256 tile.  Each CTA loads its 128 rows of A and its 128 rows of B
+//          (32 KB per 64-wide k-block, 6 stages); the leader CTA issues
+//          tcgen05.mma.cta_group::2, which reads both CTAs' shared memory, and
+//          each CTA's tensor memory receives its 128 rows of the accumulator.
+//          Operand traffic L2 -> SM per flop is 2/3 of the single-CTA form.
+//   single one CTA owns a 128x256 tile (48 KB per k-block, 4 stages); used for
+//          row fragments.
 //
 // Warp roles (192 threads, 1 CTA per SM): warp 0 = TMA producer (one lane),
 // warp 1 = tensor-memory allocation + MMA issue (one lane), warps 2..5 =
-// epilogue (warp w reads TMEM lanes 32*(w%4)..+31).  A 4-stage shared-memory
-// ring feeds the tensor core; two 256-column TMEM accumulators let the
-// epilogue of tile i overlap the main loop of tile i+1.  Every wait is bounded.
+// epilogue (warp w reads TMEM lanes 32*(w%4)..+31).  Two 256-column TMEM
+// accumulators let the epilogue of tile i overlap the main loop of tile i+1.
+// Every wait is bounded and reports COMPASS_ERR_TIMEOUT instead of hanging.
 #include "internal.h"
 #include "ptx_sm100.cuh"
 
@@ -27,17 +35,25 @@ using namespace ptx;
 
 namespace {
 
-constexpr int kStages = 4;
 constexpr int kThreads = 192;
-constexpr int kAStageBytes = BM * BK * 2;     // 16 KB
-constexpr int kBStageBytes = BN * BK * 2;     // 32 KB
-constexpr int kStageBytes = kAStageBytes + kBStageBytes;
 constexpr uint32_t kTmemCols = 512;           // two BN-column FP32 accumulators
 constexpr int kEpilogueWarps = 4;
+constexpr int kMaxStages = 6;
+
+template <bool kPair>
+struct Cfg {
+  static constexpr int kStages = kPair ? 6 : 4;
+  static constexpr int kATileBytes = BM * BK * 2;                 // 128 rows of A
+  static constexpr int kBRows = kPair ? BN / 2 : BN;              // rows of B this CTA loads
+  static constexpr int kBTileBytes = kBRows * BK * 2;
+  static constexpr int kStageBytes = kATileBytes + kBTileBytes;   // per CTA
+  static constexpr int kTileRows = kPair ? 2 * BM : BM;           // rows of one scheduling tile
+  static constexpr uint32_t kFullTxBytes = kPair ? 2 * kStageBytes : kStageBytes;
+};
 
 struct Control {
-  uint64_t full[kStages];
-  uint64_t empty[kStages];
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
   uint64_t drain;
@@ -45,7 +61,10 @@ struct Control {
   int abort;
 };
 
-constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + size_t(kStages) * kStageBytes + sizeof(Control);
+template <bool kPair>
+constexpr size_t smem_bytes() {
+  return 1024 /*alignment slack*/ + size_t(Cfg<kPair>::kStages) * Cfg<kPair>::kStageBytes + sizeof(Control);
+}
 
 __device__ __forceinline__ void report_timeout(const GemmParams& p, Control* ctl, int site, int tile) {
   *reinterpret_cast<volatile int*>(&ctl->abort) = 1;
@@ -87,36 +106,53 @@ __device__ __forceinline__ TileCoord decode_tile(const GemmParams& p, int t) {
   return c;
 }
 
+template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+  using C = Cfg<kPair>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   uint8_t* smem = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);   // 128B-swizzle tiles need 1024-byte alignment
   uint8_t* smem_a = smem;
-  uint8_t* smem_b = smem + kStages * kAStageBytes;
-  Control* ctl = reinterpret_cast<Control*>(smem + kStages * kStageBytes);
+  uint8_t* smem_b = smem + C::kStages * C::kATileBytes;
+  Control* ctl = reinterpret_cast<Control*>(smem + C::kStages * C::kStageBytes);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t cta_rank = kPair ? cluster_ctarank() : 0u;    // 0 = leader of the pair
+  const bool leader = cta_rank == 0;
+  // work units: clusters in pair mode, CTAs otherwise
+  const int unit = kPair ? int(blockIdx.x >> 1) : int(blockIdx.x);
+  const int n_units = kPair ? int(gridDim.x >> 1) : int(gridDim.x);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&ctl->full[s], 1);
       mbar_init(&ctl->empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&ctl->acc_full[b], 1);
-      mbar_init(&ctl->acc_empty[b], kEpilogueWarps);
+      mbar_init(&ctl->acc_empty[b], kPair ? 2 * kEpilogueWarps : kEpilogueWarps);
     }
     mbar_init(&ctl->drain, 1);
     ctl->abort = 0;
     fence_mbar_init();
   }
   if (warp == 1) {
-    tmem_alloc(&ctl->tmem_base, kTmemCols);
-    tmem_relinquish();
+    if (kPair) {
+      tmem_alloc_pair(&ctl->tmem_base, kTmemCols);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(&ctl->tmem_base, kTmemCols);
+      tmem_relinquish();
+    }
   }
   tc_fence_before_sync();
   __syncthreads();
+  if (kPair) {
+    // both CTAs' barriers and tensor memory exist before either CTA signals the other
+    cluster_arrive();
+    cluster_wait();
+  }
   tc_fence_after_sync();
   const uint32_t tmem_base = ctl->tmem_base;
 
@@ -129,11 +165,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       uint32_t phase = 0;
       uint32_t issued = 0;
       bool ok = true;
-      for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x) {
+      for (int t = unit; ok && t < p.total_tiles; t += n_units) {
         const TileCoord tc = decode_tile(p, t);
         const BlockDesc& b = p.blocks[tc.blk];
-        const int a_row = b.a_row0 + tc.mt * BM;
-        const int b_row = tc.nt * BN;
+        const int a_row = b.a_row0 + tc.mt * C::kTileRows + int(cta_rank) * BM;
+        const int b_row = tc.nt * BN + int(cta_rank) * C::kBRows;
         for (int seg = 0; ok && seg < p.n_seg; ++seg) {
           const int am = (p.n_seg > 1) ? p.seg_rank[tc.blk][seg] : b.a_map;
           const int bm = (p.n_seg > 1) ? am : b.b_map;
@@ -142,11 +178,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
               ok = false;
               break;
             }
-            mbar_arrive_expect_tx(&ctl->full[stage], kStageBytes);
-            tma_load_2d(smem_a + stage * kAStageBytes, &p.a_maps[am], &ctl->full[stage], kb * BK, a_row);
-            tma_load_2d(smem_b + stage * kBStageBytes, &p.b_maps[bm], &ctl->full[stage], kb * BK, b_row);
+            if (kPair) {
+              // both CTAs' loads complete on the leader's barrier, which expects the bytes of both
+              const uint32_t full_addr = map_to_cta(smem_u32(&ctl->full[stage]), 0);
+              if (leader) mbar_arrive_expect_tx(&ctl->full[stage], C::kFullTxBytes);
+              tma_load_2d_pair(smem_a + stage * C::kATileBytes, &p.a_maps[am], full_addr, kb * BK, a_row);
+              tma_load_2d_pair(smem_b + stage * C::kBTileBytes, &p.b_maps[bm], full_addr, kb * BK, b_row);
+            } else {
+              mbar_arrive_expect_tx(&ctl->full[stage], C::kFullTxBytes);
+              tma_load_2d(smem_a + stage * C::kATileBytes, &p.a_maps[am], &ctl->full[stage], kb * BK, a_row);
+              tma_load_2d(smem_b + stage * C::kBTileBytes, &p.b_maps[bm], &ctl->full[stage], kb * BK, b_row);
+            }
             ++issued;
-            if (++stage == kStages) {
+            if (++stage == C::kStages) {
               stage = 0;
               phase ^= 1u;
             }
@@ -154,23 +198,28 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         }
       }
       // Do not leave the CTA while bulk copies may still be writing shared
-      // memory: the most recent fill of every stage must have landed.
-      const uint32_t outstanding = issued < uint32_t(kStages) ? issued : uint32_t(kStages);
+      // memory: wait until the last fill of every stage has been consumed
+      // (pair: the leader's barrier tracks both CTAs' copies) or has landed.
+      const uint32_t outstanding = issued < uint32_t(C::kStages) ? issued : uint32_t(C::kStages);
       for (uint32_t i = 0; i < outstanding; ++i) {
-        stage = (stage == 0) ? kStages - 1 : stage - 1;
-        if (stage == kStages - 1) phase ^= 1u;
-        if (!wait_bounded(&ctl->full[stage], phase, ctl, p, WAIT_DRAIN, -1)) break;
+        stage = (stage == 0) ? C::kStages - 1 : stage - 1;
+        if (stage == C::kStages - 1) phase ^= 1u;
+        if (kPair) {
+          if (!wait_bounded(&ctl->empty[stage], phase, ctl, p, WAIT_DRAIN, -1)) break;
+        } else {
+          if (!wait_bounded(&ctl->full[stage], phase, ctl, p, WAIT_DRAIN, -1)) break;
+        }
       }
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16_f32(BM, BN);
+    if (lane == 0 && leader) {
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(kPair ? 2 * BM : BM, BN);
       int stage = 0;
       uint32_t phase = 0;
       uint32_t it = 0;
       bool ok = true;
-      for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++it) {
+      for (int t = unit; ok && t < p.total_tiles; t += n_units, ++it) {
         const uint32_t buf = it & 1u;
         const uint32_t acc_phase = (it >> 1) & 1u;
         if (!wait_bounded(&ctl->acc_empty[buf], acc_phase ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
@@ -183,42 +232,50 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             break;
           }
           tc_fence_after_sync();
-          const uint64_t da = umma_smem_desc_sw128(smem_u32(smem_a + stage * kAStageBytes));
-          const uint64_t db = umma_smem_desc_sw128(smem_u32(smem_b + stage * kBStageBytes));
+          const uint64_t da = umma_smem_desc_sw128(smem_u32(smem_a + stage * C::kATileBytes));
+          const uint64_t db = umma_smem_desc_sw128(smem_u32(smem_b + stage * C::kBTileBytes));
           const int ksteps = (kb_in_seg == p.kb_per_seg - 1) ? p.tail_ksteps : BK / UMMA_K;
           for (int k = 0; k < ksteps; ++k) {
             // advance 16 elements = 32 bytes inside the 128-byte swizzle row: +2 in the address field
-            umma_bf16(d_tmem, da + uint64_t(k * 2), db + uint64_t(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+            const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
+            if (kPair) umma_bf16_pair(d_tmem, da + uint64_t(k * 2), db + uint64_t(k * 2), idesc, acc);
+            else umma_bf16(d_tmem, da + uint64_t(k * 2), db + uint64_t(k * 2), idesc, acc);
           }
-          umma_commit(&ctl->empty[stage]);       // stage reusable once these MMAs have read it
+          // the stage is reusable (in both CTAs) once these MMAs have read it
+          if (kPair) umma_commit_pair(&ctl->empty[stage], 0x3);
+          else umma_commit(&ctl->empty[stage]);
           if (++kb_in_seg == p.kb_per_seg) kb_in_seg = 0;
-          if (++stage == kStages) {
+          if (++stage == C::kStages) {
             stage = 0;
             phase ^= 1u;
           }
         }
-        if (ok) umma_commit(&ctl->acc_full[buf]);   // accumulator complete
+        if (ok) {   // accumulator complete: wake the epilogue (of both CTAs)
+          if (kPair) umma_commit_pair(&ctl->acc_full[buf], 0x3);
+          else umma_commit(&ctl->acc_full[buf]);
+        }
       }
       if (*reinterpret_cast<volatile int*>(&ctl->abort)) {
         // Gave up somewhere: wait for whatever the tensor core still has in
         // flight before tensor memory is released.
-        umma_commit(&ctl->drain);
+        if (kPair) umma_commit_pair(&ctl->drain, 0x1);
+        else umma_commit(&ctl->drain);
         wait_bounded(&ctl->drain, 0, ctl, p, WAIT_DRAIN, -2);
       }
     }
   } else {
     // ---------------------------------------------------------------- epilogue
     const int quarter = warp & 3;               // TMEM lanes this warp may touch
-    const int row_in_tile = quarter * 32 + lane;
+    const int row_in_tile = int(cta_rank) * BM + quarter * 32 + lane;
     uint32_t it = 0;
-    for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++it) {
+    for (int t = unit; t < p.total_tiles; t += n_units, ++it) {
       const uint32_t buf = it & 1u;
       const uint32_t acc_phase = (it >> 1) & 1u;
       if (!wait_bounded(&ctl->acc_full[buf], acc_phase, ctl, p, WAIT_ACC_FULL, t)) break;
       tc_fence_after_sync();
       const TileCoord tc = decode_tile(p, t);
       const BlockDesc& b = p.blocks[tc.blk];
-      const int row_in_block = tc.mt * BM + row_in_tile;
+      const int row_in_block = tc.mt * C::kTileRows + row_in_tile;
       const bool row_ok = row_in_block < p.rows_per_block;
       const int ncols = min(BN, p.N - tc.nt * BN);
       const int nchunks = (ncols + 31) >> 5;
@@ -229,10 +286,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         tmem_ld_32x32b_x32(taddr + c * 32, v);
         tmem_ld_wait();
         if (c == nchunks - 1) {
-          // accumulator fully copied to registers: hand it back to the MMA warp
+          // accumulator fully copied to registers: hand it back to the MMA issuer
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&ctl->acc_empty[buf]);
+          if (lane == 0) {
+            if (kPair) mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->acc_empty[buf]), 0));
+            else mbar_arrive(&ctl->acc_empty[buf]);
+          }
         }
         if (row_ok) {
 #pragma unroll
@@ -253,9 +313,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 
   tc_fence_before_sync();
   __syncthreads();
+  if (kPair) {
+    // the peer may still signal this CTA's barriers or read its shared memory
+    cluster_arrive();
+    cluster_wait();
+  }
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if (kPair) tmem_dealloc_pair(tmem_base, kTmemCols);
+    else tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -294,16 +360,58 @@ bool encode_kmajor(CUtensorMap* map, const void* ptr, int64_t rows, int64_t K, i
   return r == CUDA_SUCCESS;
 }
 
+struct DeviceInfo {
+  int num_sms = 0;
+  int max_pairs = 0;     // co-resident clusters of two CTAs of the pair kernel
+  bool ready = false;
+};
+
+int device_info(DeviceInfo** out) {
+  static DeviceInfo info;
+  if (!info.ready) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaDeviceGetAttribute(&info.num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<false>()));
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<true>()));
+    if (e != cudaSuccess) return record_cuda_error(e);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(info.num_sms / 2 * 2));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_bytes<true>();
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    e = cudaOccupancyMaxActiveClusters(&clusters, gemm_kernel<true>, &cfg);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    info.max_pairs = clusters;
+    info.ready = true;
+  }
+  *out = &info;
+  return COMPASS_OK;
+}
+
 }  // namespace
 
-size_t gemm_smem_bytes() { return kSmemBytes; }
+size_t gemm_smem_bytes() { return smem_bytes<true>() > smem_bytes<false>() ? smem_bytes<true>() : smem_bytes<false>(); }
 
 int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   static thread_local GemmParams p;
+  const bool pair = L.mode == GEMM_MODE_PAIR || (L.mode == GEMM_MODE_AUTO && L.rows_per_block >= 2 * BM);
+  const int tile_rows = pair ? 2 * BM : BM;
+  const int b_box_rows = pair ? BN / 2 : BN;
   for (int i = 0; i < L.n_a; ++i)
     if (!encode_kmajor(&p.a_maps[i], L.a_ptr[i], L.a_rows, L.K, BM)) return record_cuda_error(cudaErrorUnknown);
   for (int i = 0; i < L.n_b; ++i)
-    if (!encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, BN)) return record_cuda_error(cudaErrorUnknown);
+    if (!encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, b_box_rows)) return record_cuda_error(cudaErrorUnknown);
   for (int i = 0; i < L.n_out; ++i) p.out[i] = static_cast<__nv_bfloat16*>(L.out_ptr[i]);
   p.ldo = L.ldo;
   p.n_blocks = L.n_blocks;
@@ -313,7 +421,7 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   p.kb_per_seg = int32_t((L.K + BK - 1) / BK);
   const int64_t k_tail = L.K - int64_t(p.kb_per_seg - 1) * BK;
   p.tail_ksteps = int32_t((k_tail + UMMA_K - 1) / UMMA_K);
-  p.tiles_m = (L.rows_per_block + BM - 1) / BM;
+  p.tiles_m = (L.rows_per_block + tile_rows - 1) / tile_rows;
   p.tiles_n = int32_t((L.N + BN - 1) / BN);
   p.total_tiles = L.n_blocks * p.tiles_m * p.tiles_n;
   p.epilogue = L.epilogue;
@@ -326,23 +434,40 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
     for (int b = 0; b < L.n_blocks; ++b)
       for (int s = 0; s < L.n_seg; ++s) p.seg_rank[b][s] = L.seg_rank[b][s];
 
-  static int num_sms = 0;
-  static bool attr_set = false;
-  if (!attr_set) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    e = cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemBytes));
-    if (e != cudaSuccess) return record_cuda_error(e);
-    attr_set = true;
-  }
+  DeviceInfo* info = nullptr;
+  int st = device_info(&info);
+  if (st != COMPASS_OK) return st;
   if (p.total_tiles <= 0) return COMPASS_OK;
-  const int grid = p.total_tiles < num_sms ? p.total_tiles : num_sms;
-  gemm_kernel<<<grid, kThreads, kSmemBytes, stream>>>(p);
+  cudaError_t e;
+  if (pair && info->max_pairs > 0) {
+    const int pairs = p.total_tiles < info->max_pairs ? p.total_tiles : info->max_pairs;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(2 * pairs));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_bytes<true>();
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, gemm_kernel<true>, p);
+  } else {
+    if (pair) {   // no room for clusters on this device: fall back to single-CTA tiles
+      p.tiles_m = (L.rows_per_block + BM - 1) / BM;
+      p.total_tiles = L.n_blocks * p.tiles_m * p.tiles_n;
+      for (int i = 0; i < L.n_b; ++i)
+        if (!encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, BN)) return record_cuda_error(cudaErrorUnknown);
+    }
+    const int grid = p.total_tiles < info->num_sms ? p.total_tiles : info->num_sms;
+    gemm_kernel<false><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);
+    e = cudaGetLastError();
+  }
   count_kernel_launch();
-  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return record_cuda_error(e);
+  e = cudaGetLastError();
   if (e != cudaSuccess) return record_cuda_error(e);
   return COMPASS_OK;
 }

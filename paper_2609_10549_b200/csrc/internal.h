@@ -52,6 +52,12 @@ struct BlockDesc {
   uint8_t pad[3];
 };
 
+enum GemmMode : int32_t {
+  GEMM_MODE_AUTO = 0,     // CTA pairs when a block has at least 256 rows
+  GEMM_MODE_SINGLE = 1,   // one CTA per 128x256 tile
+  GEMM_MODE_PAIR = 2,     // two CTAs per 256x256 tile
+};
+
 enum EpilogueMode : int32_t {
   EPI_STORE = 0,      // round to BF16 and store
   EPI_RING_RMW = 1,   // ordered accumulate into the output in ring order
@@ -92,6 +98,7 @@ struct GemmLaunch {
   int n_seg = 1;
   int rows_per_block = 0;
   int epilogue = EPI_STORE;
+  int mode = GEMM_MODE_AUTO;
   int last_step = 0;
   int n_blocks = 0;
   BlockDesc blocks[kMaxBlocks];
