@@ -67,6 +67,16 @@ enum { COMPASS_DTYPE_BF16 = 0 };
  *     writes the BF16 result).  Needs tile counters in the workspace. */
 enum { COMPASS_RS_SEGMENTED_K = 0, COMPASS_RS_RING_RMW = 1 };
 enum { COMPASS_STRATEGY_INTRAFUSION = 0, COMPASS_STRATEGY_INTERDECOM = 1 };
+/* Launch order of the fused kernels.  Every rank's tiles are always issued in
+ * that rank's schedule order (step ascending, ring 0 before ring 1).  What the
+ * emulation is free to choose is how the P ranks' sequences are merged on the
+ * one GPU:
+ *   RANK_MAJOR: rank 0's whole sequence, then rank 1's, ... (a rank's weight
+ *     shard stays in L2 while it is used; default);
+ *   STEP_MAJOR: all ranks advance in lockstep: step 0 of every rank, then
+ *     step 1, ... (what P GPUs running concurrently would do).
+ * The ring read-modify-write variant always uses STEP_MAJOR. */
+enum { COMPASS_ORDER_RANK_MAJOR = 0, COMPASS_ORDER_STEP_MAJOR = 1 };
 /* selectors for compass_workspace_bytes */
 enum { COMPASS_WS_FUSED = 0, COMPASS_WS_DECOMP = 1 };
 
@@ -80,6 +90,8 @@ typedef struct compass_problem {
   int64_t M, N, K;
   int32_t dtype;       /* COMPASS_DTYPE_BF16 */
   int32_t rs_variant;  /* COMPASS_RS_* (GEMM+ReduceScatter only) */
+  int32_t order;       /* COMPASS_ORDER_* : how the P logical ranks share the one GPU */
+  int32_t reserved;    /* must be 0 */
 } compass_problem;
 
 /* One line of the ring chunk schedule (Section III-B).  `part` = rings*chunk +

@@ -20,6 +20,7 @@ OP_AG_GEMM, OP_GEMM_RS = 0, 1
 DTYPE_BF16 = 0
 RS_SEGMENTED_K, RS_RING_RMW = 0, 1
 STRATEGY_INTRAFUSION, STRATEGY_INTERDECOM = 0, 1
+ORDER_RANK_MAJOR, ORDER_STEP_MAJOR = 0, 1
 WS_FUSED, WS_DECOMP = 0, 1
 MAX_P = 16
 STATUS_BYTES = 256
@@ -43,7 +44,7 @@ class CompassError(RuntimeError):
 class Problem(C.Structure):
     _fields_ = [("op", C.c_int32), ("P", C.c_int32), ("rings", C.c_int32), ("d", C.c_int32),
                 ("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64),
-                ("dtype", C.c_int32), ("rs_variant", C.c_int32)]
+                ("dtype", C.c_int32), ("rs_variant", C.c_int32), ("order", C.c_int32), ("reserved", C.c_int32)]
 
 
 class SchedEntry(C.Structure):
@@ -122,8 +123,9 @@ def _check(status: int, where: str) -> None:
 
 
 def make_problem(op: int, P: int, M: int, N: int, K: int, rings: int = 2, d: int = 1,
-                 rs_variant: int = RS_SEGMENTED_K, dtype: int = DTYPE_BF16) -> Problem:
-    return Problem(op=op, P=P, rings=rings, d=d, M=M, N=N, K=K, dtype=dtype, rs_variant=rs_variant)
+                 rs_variant: int = RS_SEGMENTED_K, dtype: int = DTYPE_BF16, order: int = ORDER_RANK_MAJOR) -> Problem:
+    return Problem(op=op, P=P, rings=rings, d=d, M=M, N=N, K=K, dtype=dtype, rs_variant=rs_variant, order=order,
+                   reserved=0)
 
 
 # ---- host-only calls -------------------------------------------------------------

@@ -24,6 +24,8 @@ int validate_problem(const compass_problem* pr, int want_op, bool need_d) {
   if (want_op >= 0 && pr->op != want_op) return COMPASS_ERR_INVALID_ARG;
   if (pr->P < 1 || (pr->rings != 1 && pr->rings != 2)) return COMPASS_ERR_INVALID_ARG;
   if (need_d && pr->d < 1) return COMPASS_ERR_INVALID_ARG;
+  if ((pr->order != COMPASS_ORDER_RANK_MAJOR && pr->order != COMPASS_ORDER_STEP_MAJOR) || pr->reserved != 0)
+    return COMPASS_ERR_INVALID_ARG;
   if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant != COMPASS_RS_SEGMENTED_K && pr->rs_variant != COMPASS_RS_RING_RMW)
     return COMPASS_ERR_INVALID_ARG;
   if (pr->dtype != COMPASS_DTYPE_BF16 || pr->P > COMPASS_MAX_P) return COMPASS_ERR_UNSUPPORTED;
@@ -78,28 +80,32 @@ void plan_ag(const compass_problem* pr, const compass_sched_entry* table, GemmLa
   L->rows_per_block = int(m / rings);
   L->epilogue = EPI_STORE;
   int n = 0;
-  for (int step = 0; step < P; ++step)
-    for (int ring = 0; ring < rings; ++ring)
-      for (int rank = 0; rank < P; ++rank) {
-        const compass_sched_entry& e = table[(size_t(rank) * P + step) * rings + ring];
-        BlockDesc& b = L->blocks[n];
-        std::memset(&b, 0, sizeof(b));
-        b.a_map = uint8_t(e.chunk);                       // read the owner's shard: gather by address
-        b.a_row0 = e.row_begin - e.chunk * int32_t(m);
-        b.b_map = uint8_t(rank);
-        b.out_idx = uint8_t(rank);
-        b.out_row0 = e.row_begin;
-        b.step = uint8_t(step);
-        b.part = uint8_t(e.part);
-        if (view) {
-          compass_plan_block& v = view[n];
-          v.rank = rank; v.step = step; v.ring = ring; v.part = e.part;
-          v.a_tensor = e.chunk; v.a_row_begin = b.a_row0;
-          v.out_tensor = rank; v.out_row_begin = b.out_row0;
-          v.rows = e.row_count;
-        }
-        ++n;
-      }
+  const bool rank_major = pr->order == COMPASS_ORDER_RANK_MAJOR;
+  const int n_entries = P * P * rings;
+  for (int i = 0; i < n_entries; ++i) {
+    // rank-major: the table's own order; step-major: step, then ring, then rank
+    const int rank = rank_major ? i / (P * rings) : i % P;
+    const int step = rank_major ? (i / rings) % P : i / (rings * P);
+    const int ring = rank_major ? i % rings : (i / P) % rings;
+    const compass_sched_entry& e = table[(size_t(rank) * P + step) * rings + ring];
+    BlockDesc& b = L->blocks[n];
+    std::memset(&b, 0, sizeof(b));
+    b.a_map = uint8_t(e.chunk);                       // read the owner's shard: gather by address
+    b.a_row0 = e.row_begin - e.chunk * int32_t(m);
+    b.b_map = uint8_t(rank);
+    b.out_idx = uint8_t(rank);
+    b.out_row0 = e.row_begin;
+    b.step = uint8_t(step);
+    b.part = uint8_t(e.part);
+    if (view) {
+      compass_plan_block& v = view[n];
+      v.rank = rank; v.step = step; v.ring = ring; v.part = e.part;
+      v.a_tensor = e.chunk; v.a_row_begin = b.a_row0;
+      v.out_tensor = rank; v.out_row_begin = b.out_row0;
+      v.rows = e.row_count;
+    }
+    ++n;
+  }
   L->n_blocks = n;
 }
 
@@ -195,7 +201,7 @@ int plan_fused(const compass_problem* pr, GemmLaunch* L, compass_plan_block* vie
   else if (pr->rs_variant == COMPASS_RS_SEGMENTED_K) plan_rs_segmented(pr, table, L, view);
   else plan_rs_ring(pr, table, L, view);
   if (view) {
-    const int per_block = tiles_of(L->rows_per_block, BM) * tiles_of(L->N, BN);
+    const int per_block = tiles_of(L->rows_per_block, gemm_tile_rows(L->mode, L->rows_per_block)) * tiles_of(L->N, BN);
     for (int i = 0; i < L->n_blocks; ++i) {
       view[i].first_tile = i * per_block;
       view[i].tile_count = per_block;

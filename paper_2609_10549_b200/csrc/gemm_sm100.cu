@@ -14,7 +14,7 @@
 // Two modes of the same kernel:
 //   pair   (default when a block has >= 256 rows): a cluster of two CTAs owns a
 //          256x256 tile.  Each CTA loads its 128 rows of A and its 128 rows of B
-//          (32 KB per 64-wide k-block, 6 stages); the leader CTA issues
+//          (64 KB per 128-wide k-stage, 3 stages); the leader CTA issues
 //          tcgen05.mma.cta_group::2, which reads both CTAs' shared memory, and
 //          each CTA's tensor memory receives its 128 rows of the accumulator.
 //          Operand traffic L2 -> SM per flop is 2/3 of the single-CTA form.
@@ -38,14 +38,23 @@ namespace {
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;           // two BN-column FP32 accumulators
 constexpr int kEpilogueWarps = 4;
-constexpr int kMaxStages = 6;
+constexpr int kMaxStages = 7;
 
 template <bool kPair>
 struct Cfg {
-  static constexpr int kStages = kPair ? 6 : 4;
-  static constexpr int kATileBytes = BM * BK * 2;                 // 128 rows of A
+  // A pipeline stage holds kAtoms k-atoms of 64 elements (one 128-byte swizzle
+  // row each).  The MMA issuer pays a fixed cost per stage (barrier wait,
+  // commit, loop) of a few hundred cycles during which the tensor core only has
+  // the queued MMAs to work on, so a stage must carry enough of them: 8 per
+  // stage keep the pipe full, 4 do not.
+  static constexpr int kAtoms = kPair ? 2 : 1;
+  static constexpr int kStageK = kAtoms * BK;
+  static constexpr int kStages = kPair ? 3 : 4;
+  static constexpr int kAAtomBytes = BM * BK * 2;                 // 128 rows of A, one atom
   static constexpr int kBRows = kPair ? BN / 2 : BN;              // rows of B this CTA loads
-  static constexpr int kBTileBytes = kBRows * BK * 2;
+  static constexpr int kBAtomBytes = kBRows * BK * 2;
+  static constexpr int kATileBytes = kAtoms * kAAtomBytes;
+  static constexpr int kBTileBytes = kAtoms * kBAtomBytes;
   static constexpr int kStageBytes = kATileBytes + kBTileBytes;   // per CTA
   static constexpr int kTileRows = kPair ? 2 * BM : BM;           // rows of one scheduling tile
   static constexpr uint32_t kFullTxBytes = kPair ? 2 * kStageBytes : kStageBytes;
@@ -165,6 +174,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       uint32_t phase = 0;
       uint32_t issued = 0;
       bool ok = true;
+      const uint64_t pol_a = make_l2_policy(p.a_hint);
+      const uint64_t pol_b = make_l2_policy(p.b_hint);
       for (int t = unit; ok && t < p.total_tiles; t += n_units) {
         const TileCoord tc = decode_tile(p, t);
         const BlockDesc& b = p.blocks[tc.blk];
@@ -178,16 +189,27 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
               ok = false;
               break;
             }
+            const int kx = kb * C::kStageK;
             if (kPair) {
               // both CTAs' loads complete on the leader's barrier, which expects the bytes of both
               const uint32_t full_addr = map_to_cta(smem_u32(&ctl->full[stage]), 0);
               if (leader) mbar_arrive_expect_tx(&ctl->full[stage], C::kFullTxBytes);
-              tma_load_2d_pair(smem_a + stage * C::kATileBytes, &p.a_maps[am], full_addr, kb * BK, a_row);
-              tma_load_2d_pair(smem_b + stage * C::kBTileBytes, &p.b_maps[bm], full_addr, kb * BK, b_row);
+#pragma unroll
+              for (int at = 0; at < C::kAtoms; ++at) {
+                tma_load_2d_pair_hint(smem_a + stage * C::kATileBytes + at * C::kAAtomBytes, &p.a_maps[am], full_addr,
+                                      kx + at * BK, a_row, pol_a);
+                tma_load_2d_pair_hint(smem_b + stage * C::kBTileBytes + at * C::kBAtomBytes, &p.b_maps[bm], full_addr,
+                                      kx + at * BK, b_row, pol_b);
+              }
             } else {
               mbar_arrive_expect_tx(&ctl->full[stage], C::kFullTxBytes);
-              tma_load_2d(smem_a + stage * C::kATileBytes, &p.a_maps[am], &ctl->full[stage], kb * BK, a_row);
-              tma_load_2d(smem_b + stage * C::kBTileBytes, &p.b_maps[bm], &ctl->full[stage], kb * BK, b_row);
+#pragma unroll
+              for (int at = 0; at < C::kAtoms; ++at) {
+                tma_load_2d_hint(smem_a + stage * C::kATileBytes + at * C::kAAtomBytes, &p.a_maps[am], &ctl->full[stage],
+                                 kx + at * BK, a_row, pol_a);
+                tma_load_2d_hint(smem_b + stage * C::kBTileBytes + at * C::kBAtomBytes, &p.b_maps[bm], &ctl->full[stage],
+                                 kx + at * BK, b_row, pol_b);
+              }
             }
             ++issued;
             if (++stage == C::kStages) {
@@ -232,14 +254,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             break;
           }
           tc_fence_after_sync();
-          const uint64_t da = umma_smem_desc_sw128(smem_u32(smem_a + stage * C::kATileBytes));
-          const uint64_t db = umma_smem_desc_sw128(smem_u32(smem_b + stage * C::kBTileBytes));
-          const int ksteps = (kb_in_seg == p.kb_per_seg - 1) ? p.tail_ksteps : BK / UMMA_K;
-          for (int k = 0; k < ksteps; ++k) {
-            // advance 16 elements = 32 bytes inside the 128-byte swizzle row: +2 in the address field
-            const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
-            if (kPair) umma_bf16_pair(d_tmem, da + uint64_t(k * 2), db + uint64_t(k * 2), idesc, acc);
-            else umma_bf16(d_tmem, da + uint64_t(k * 2), db + uint64_t(k * 2), idesc, acc);
+          const uint32_t a_base = smem_u32(smem_a + stage * C::kATileBytes);
+          const uint32_t b_base = smem_u32(smem_b + stage * C::kBTileBytes);
+          const int ksteps = (kb_in_seg == p.kb_per_seg - 1) ? p.tail_ksteps : C::kStageK / UMMA_K;
+          for (int ks = 0; ks < ksteps; ++ks) {
+            // a 64-element atom holds 4 steps of 16 elements = 32 bytes each: +2 in the descriptor's address field
+            const int at = ks >> 2, k = ks & 3;
+            const uint64_t da = umma_smem_desc_sw128(a_base + at * C::kAAtomBytes) + uint64_t(k * 2);
+            const uint64_t db = umma_smem_desc_sw128(b_base + at * C::kBAtomBytes) + uint64_t(k * 2);
+            const uint32_t acc = (kb | ks) != 0 ? 1u : 0u;
+            if (kPair) umma_bf16_pair(d_tmem, da, db, idesc, acc);
+            else umma_bf16(d_tmem, da, db, idesc, acc);
           }
           // the stage is reusable (in both CTAs) once these MMAs have read it
           if (kPair) umma_commit_pair(&ctl->empty[stage], 0x3);
@@ -403,10 +428,15 @@ int device_info(DeviceInfo** out) {
 
 size_t gemm_smem_bytes() { return smem_bytes<true>() > smem_bytes<false>() ? smem_bytes<true>() : smem_bytes<false>(); }
 
+int gemm_tile_rows(int mode, int rows_per_block) {
+  const bool pair = mode == GEMM_MODE_PAIR || (mode == GEMM_MODE_AUTO && rows_per_block >= 2 * BM);
+  return pair ? 2 * BM : BM;
+}
+
 int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   static thread_local GemmParams p;
-  const bool pair = L.mode == GEMM_MODE_PAIR || (L.mode == GEMM_MODE_AUTO && L.rows_per_block >= 2 * BM);
-  const int tile_rows = pair ? 2 * BM : BM;
+  const int tile_rows = gemm_tile_rows(L.mode, L.rows_per_block);
+  const bool pair = tile_rows == 2 * BM;
   const int b_box_rows = pair ? BN / 2 : BN;
   for (int i = 0; i < L.n_a; ++i)
     if (!encode_kmajor(&p.a_maps[i], L.a_ptr[i], L.a_rows, L.K, BM)) return record_cuda_error(cudaErrorUnknown);
@@ -418,8 +448,9 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   p.rows_per_block = L.rows_per_block;
   p.N = int32_t(L.N);
   p.n_seg = L.n_seg;
-  p.kb_per_seg = int32_t((L.K + BK - 1) / BK);
-  const int64_t k_tail = L.K - int64_t(p.kb_per_seg - 1) * BK;
+  const int stage_k = pair ? 2 * BK : BK;      // Cfg<pair>::kStageK
+  p.kb_per_seg = int32_t((L.K + stage_k - 1) / stage_k);
+  const int64_t k_tail = L.K - int64_t(p.kb_per_seg - 1) * stage_k;
   p.tail_ksteps = int32_t((k_tail + UMMA_K - 1) / UMMA_K);
   p.tiles_m = (L.rows_per_block + tile_rows - 1) / tile_rows;
   p.tiles_n = int32_t((L.N + BN - 1) / BN);
@@ -427,6 +458,9 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   p.epilogue = L.epilogue;
   p.last_step = L.last_step;
   p.wait_limit_us = 2000000u;
+  p.a_hint = L.a_hint;
+  p.b_hint = L.b_hint;
+
   p.status = L.status;
   p.tile_counters = L.tile_counters;
   for (int b = 0; b < L.n_blocks; ++b) p.blocks[b] = L.blocks[b];
@@ -458,6 +492,8 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
     if (pair) {   // no room for clusters on this device: fall back to single-CTA tiles
       p.tiles_m = (L.rows_per_block + BM - 1) / BM;
       p.total_tiles = L.n_blocks * p.tiles_m * p.tiles_n;
+      p.kb_per_seg = int32_t((L.K + BK - 1) / BK);
+      p.tail_ksteps = int32_t((L.K - int64_t(p.kb_per_seg - 1) * BK + UMMA_K - 1) / UMMA_K);
       for (int i = 0; i < L.n_b; ++i)
         if (!encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, BN)) return record_cuda_error(cudaErrorUnknown);
     }

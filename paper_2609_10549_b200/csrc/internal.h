@@ -72,13 +72,14 @@ struct GemmParams {
   int32_t rows_per_block;
   int32_t N;               // output columns
   int32_t n_seg;           // K segments accumulated into one tile (1, or P for segmented-K reduce)
-  int32_t kb_per_seg;      // k-blocks of BK per segment (last one may be partial)
-  int32_t tail_ksteps;     // UMMA_K steps in the last k-block of a segment (1..BK/UMMA_K)
+  int32_t kb_per_seg;      // k-stages per segment (last one may be partial)
+  int32_t tail_ksteps;     // UMMA_K steps in the last k-stage of a segment
   int32_t tiles_m, tiles_n;
   int32_t total_tiles;
   int32_t epilogue;        // EpilogueMode
   int32_t last_step;       // ring RMW: step index of the final contributor (P-1)
   uint32_t wait_limit_us;  // bound of every device-side wait
+  int32_t a_hint, b_hint;  // L2 eviction priority of the A / B tile loads (ptx::L2Hint)
   StatusBlock* status;
   int32_t* tile_counters;  // ring RMW only
   uint8_t seg_rank[kMaxSegBlocks][kMaxP];   // segmented-K: tensor index of segment s of block b
@@ -99,6 +100,7 @@ struct GemmLaunch {
   int rows_per_block = 0;
   int epilogue = EPI_STORE;
   int mode = GEMM_MODE_AUTO;
+  int a_hint = 0, b_hint = 0;
   int last_step = 0;
   int n_blocks = 0;
   BlockDesc blocks[kMaxBlocks];
@@ -110,6 +112,7 @@ struct GemmLaunch {
 // gemm_sm100.cu
 int launch_gemm(const GemmLaunch& launch, cudaStream_t stream);
 size_t gemm_smem_bytes();
+int gemm_tile_rows(int mode, int rows_per_block);   // rows of one scheduling tile: 256 (CTA pair) or 128
 
 // aux_kernels.cu
 int launch_reduce_partials(const void* const* partial, int P, void* const* out, int64_t m, int64_t N,

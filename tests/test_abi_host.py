@@ -30,7 +30,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_layouts_match_the_header():
-    assert C.sizeof(api.Problem) == 4 * 4 + 3 * 8 + 2 * 4
+    assert C.sizeof(api.Problem) == 4 * 4 + 3 * 8 + 4 * 4
     assert C.sizeof(api.SchedEntry) == 32
     assert C.sizeof(api.Calib) == 64
     assert C.sizeof(api.Choice) == 8 + 6 * 8
@@ -165,6 +165,9 @@ def test_problem_validation_codes():
     assert _codes(api.make_problem(**ok), 7)[0] == api.ERR_INVALID_ARG
     rs = api.make_problem(OP_GEMM_RS, 8, 8192, 4096, 1376, rs_variant=5)
     assert _codes(rs)[0] == api.ERR_INVALID_ARG
+    assert _codes(api.make_problem(**ok, order=2))[0] == api.ERR_INVALID_ARG
+    res = api.make_problem(**ok); res.reserved = 1
+    assert _codes(res)[0] == api.ERR_INVALID_ARG
 
 
 def test_workspace_sizes():
@@ -204,10 +207,11 @@ def test_fused_calls_refuse_bad_arguments_before_touching_the_gpu():
     assert api.status_string(api.ERR_TIMEOUT) == "device-side wait timed out"
 
 
+@pytest.mark.parametrize("order", [api.ORDER_RANK_MAJOR, api.ORDER_STEP_MAJOR])
 @pytest.mark.parametrize("P,rings", [(1, 2), (2, 2), (4, 2), (8, 2), (4, 1), (16, 2)])
-def test_ag_launch_plan_keeps_each_ranks_schedule_order(P, rings):
+def test_ag_launch_plan_keeps_each_ranks_schedule_order(P, rings, order):
     M, N, K = P * 512, 1024, 256
-    pr = api.make_problem(OP_AG_GEMM, P, M, N, K, rings=rings)
+    pr = api.make_problem(OP_AG_GEMM, P, M, N, K, rings=rings, order=order)
     plan = api.compass_launch_plan(pr)
     table = oracle_schedule(OP_AG_GEMM, P, rings, M)
     assert len(plan) == len(table)
@@ -220,11 +224,15 @@ def test_ag_launch_plan_keeps_each_ranks_schedule_order(P, rings):
             # the A rows are read from the shard of the chunk's owner: gather by address
             assert b.a_tensor == e[4] and b.a_row_begin == e[6] - e[4] * m and b.rows == e[7]
             assert b.out_tensor == r and b.out_row_begin == e[6]
-    # launch order is step-major and tiles are consecutive
-    assert [b.step for b in plan] == sorted(b.step for b in plan)
+    # how the ranks' sequences are merged, and tiles are consecutive
+    if order == api.ORDER_STEP_MAJOR:
+        assert [b.step for b in plan] == sorted(b.step for b in plan)
+    else:
+        assert [b.rank for b in plan] == sorted(b.rank for b in plan)
+    tile_rows = 256 if M // P // rings >= 256 else 128
     first = 0
     for b in plan:
-        assert b.first_tile == first and b.tile_count == math.ceil(b.rows / 128) * math.ceil(N / 256)
+        assert b.first_tile == first and b.tile_count == math.ceil(b.rows / tile_rows) * math.ceil(N / 256)
         first += b.tile_count
 
 
