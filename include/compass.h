@@ -41,6 +41,8 @@ extern "C" {
 
 #define COMPASS_MAX_P 16            /* largest tensor-parallel size accepted */
 #define COMPASS_STATUS_BYTES 256    /* status block at the start of every workspace */
+/* size of the built-in device array behind compass_gemm_rs_sequential_noalloc (32 MiB) */
+#define COMPASS_NOALLOC_SCRATCH_BYTES (32u * 1024u * 1024u)
 
 typedef enum compass_status {
   COMPASS_OK = 0,
@@ -51,7 +53,9 @@ typedef enum compass_status {
                                        (rows must be a multiple of 16 bytes for the tensor-map loads) */
   COMPASS_ERR_BUFFER_TOO_SMALL = 5, /* schedule capacity or workspace bytes */
   COMPASS_ERR_CUDA = 6,             /* a CUDA call failed; see compass_last_cuda_error() */
-  COMPASS_ERR_TIMEOUT = 7           /* a bounded device-side wait gave up (from compass_read_status) */
+  COMPASS_ERR_TIMEOUT = 7,          /* a bounded device-side wait gave up (from compass_read_status) */
+  COMPASS_ERR_SCRATCH_LIMIT = 8     /* the problem needs more scratch than the built-in array of the
+                                       no-allocation entry point holds */
 } compass_status;
 
 enum { COMPASS_OP_AG_GEMM = 0, COMPASS_OP_GEMM_RS = 1 };
@@ -230,6 +234,36 @@ int compass_launch_plan(const compass_problem* problem, compass_plan_block* out,
 int compass_fused_host(const compass_problem* problem, const void* const* A_host, const void* const* B_host,
                        void* const* out_host, void* staging, size_t staging_bytes, size_t* staging_bytes_needed,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+/* ---- no-allocation variant (the paper has no counterpart) -------------------
+ * GEMM+ReduceScatter in its sequential form -- one GEMM that writes every
+ * rank's BF16 partial product, then the reduce kernel that sums the P partials
+ * in FP32 into the owners' rows (the same result, bit for bit, as
+ * compass_decomp with d = 1) -- for callers that cannot hand the library a
+ * workspace: a process whose device memory was all given out before this call
+ * (a server or job started with a fixed memory budget that fills the GPU, a
+ * plug-in inside another framework's memory pool), where a cudaMalloc for the
+ * partials would fail, fragment the pool or stall every stream, or a
+ * latency-critical loop that cannot afford the device-wide synchronisation of
+ * cudaMalloc/cudaFree.  The caller passes only inputs and outputs:
+ *   A: P device pointers [M x K];  B: P device pointers [N x K];
+ *   Out: P device pointers [M/P x N] (every element is written).
+ * The scratch (status block + P partial products of M*N BF16 each) is a
+ * built-in device array of COMPASS_NOALLOC_SCRATCH_BYTES; every GPU on which
+ * the library is loaded holds it until the process exits.  A problem with
+ * 256 + P * M * N * 2 bytes (each partial rounded up to 256 bytes) beyond that
+ * size is refused with COMPASS_ERR_SCRATCH_LIMIT.  The call allocates nothing:
+ * no cudaMalloc, no cudaFree, no allocating library routine.
+ * The first call on a device looks up the array's device address (once per
+ * device, with that device current); make that first call before any stream
+ * capture begins.  All calls on a GPU share the array, which keeps what the
+ * previous call left in it (the status block is cleared at the start of every
+ * call; the partials are overwritten before they are read): calls ordered on
+ * one stream are fine, calls that overlap on the GPU race and give undefined
+ * results.  A device-side wait that gives up is recorded inside the array and
+ * cannot be read back through this entry point. */
+int compass_gemm_rs_sequential_noalloc(const compass_problem* problem, const void* const* A, const void* const* B,
+                                       void* const* Out, void* cuda_stream);
+
 const char* compass_status_string(int status);
 int compass_last_cuda_error(void);
 /* Number of kernels this library has launched since it was loaded. */

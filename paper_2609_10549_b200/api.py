@@ -16,6 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libcompass.so")
 
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = range(8)
+ERR_SCRATCH_LIMIT = 8
+NOALLOC_SCRATCH_BYTES = 32 * 1024 * 1024
 OP_AG_GEMM, OP_GEMM_RS = 0, 1
 DTYPE_BF16 = 0
 RS_SEGMENTED_K, RS_RING_RMW = 0, 1
@@ -31,7 +33,7 @@ EXPORTS = (
     "compass_model_decomp_time", "compass_model_optimal_degree", "compass_model_fusion_time",
     "compass_calib_fit_decomp", "compass_calib_fit_fusion", "compass_workspace_bytes", "compass_workspace_init",
     "compass_read_status", "compass_launch_plan", "compass_fused_host", "compass_status_string",
-    "compass_last_cuda_error", "compass_kernel_launch_count",
+    "compass_last_cuda_error", "compass_kernel_launch_count", "compass_gemm_rs_sequential_noalloc",
 )
 
 
@@ -97,6 +99,7 @@ def lib() -> C.CDLL:
         L.compass_launch_plan.argtypes = [C.POINTER(Problem), C.POINTER(PlanBlock), C.c_size_t, C.POINTER(C.c_size_t)]
         L.compass_fused_host.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t),
                                          C.c_void_p, C.c_size_t, C.c_void_p]
+        L.compass_gemm_rs_sequential_noalloc.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p]
         L.compass_status_string.argtypes = [C.c_int]
         L.compass_status_string.restype = C.c_char_p
         L.compass_last_cuda_error.restype = C.c_int
@@ -252,6 +255,15 @@ def compass_decomp(problem: Problem, A: Sequence, B: Sequence, out: Sequence, wo
     sp = _stream_handle(stream_copy) if stream_copy is not None else sc
     _check(lib().compass_decomp(C.byref(problem), _ptr_array(A), _ptr_array(B), _ptr_array(out), p, n, sc, sp),
            "compass_decomp")
+
+
+def compass_gemm_rs_sequential_noalloc(problem: Problem, A: Sequence, B: Sequence, Out: Sequence, stream=None) -> None:
+    """GEMM+ReduceScatter (sequential form) whose scratch is the library's built-in
+    device array: for callers that cannot allocate or pass a workspace (all device
+    memory already handed out, or no tolerance for cudaMalloc's device-wide sync).
+    Refuses problems needing more than NOALLOC_SCRATCH_BYTES."""
+    _check(lib().compass_gemm_rs_sequential_noalloc(C.byref(problem), _ptr_array(A), _ptr_array(B), _ptr_array(Out),
+                                                    _stream_handle(stream)), "compass_gemm_rs_sequential_noalloc")
 
 
 def compass_fused_host_bytes(problem: Problem) -> int:

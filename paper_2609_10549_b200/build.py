@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcompass.so")
-SOURCES = ["api.cu", "gemm_sm100.cu", "aux_kernels.cu", "schedule.cpp", "models.cpp"]
+SOURCES = ["api.cu", "gemm_sm100.cu", "aux_kernels.cu", "no_alloc.cu", "schedule.cpp", "models.cpp"]
 
 
 def _nvcc() -> str:

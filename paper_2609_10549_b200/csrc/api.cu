@@ -504,6 +504,7 @@ extern "C" const char* compass_status_string(int status) {
     case COMPASS_ERR_BUFFER_TOO_SMALL: return "buffer too small";
     case COMPASS_ERR_CUDA: return "CUDA call failed";
     case COMPASS_ERR_TIMEOUT: return "device-side wait timed out";
+    case COMPASS_ERR_SCRATCH_LIMIT: return "problem exceeds the built-in scratch array of the no-allocation entry point";
     default: return "unknown status";
   }
 }
