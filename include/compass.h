@@ -66,9 +66,12 @@ enum { COMPASS_DTYPE_BF16 = 0 };
  *     BF16 rounding.
  *   RING_RMW: every rank's partial tile is produced separately in that rank's
  *     schedule order and added into the owner's rows in ring order by a
- *     vectorised read-modify-write in the GEMM epilogue (the running sum is
- *     kept in FP32 in the workspace; the owner's contribution, scheduled last,
- *     writes the BF16 result).  Needs tile counters in the workspace. */
+ *     vectorised read-modify-write in the GEMM epilogue.  The running sum lives
+ *     in the BF16 output rows (what a BF16 ring transfer would carry), so the
+ *     result is rounded once per contributor; the owner's contribution,
+ *     scheduled last, completes it.  Needs one int32 counter per output tile in
+ *     the workspace (zero before the first call; every call leaves them zero,
+ *     unless it reported COMPASS_ERR_TIMEOUT: then re-initialise the workspace). */
 enum { COMPASS_RS_SEGMENTED_K = 0, COMPASS_RS_RING_RMW = 1 };
 enum { COMPASS_STRATEGY_INTRAFUSION = 0, COMPASS_STRATEGY_INTERDECOM = 1 };
 /* Launch order of the fused kernels.  Every rank's tiles are always issued in
@@ -264,6 +267,10 @@ int compass_fused_host(const compass_problem* problem, const void* const* A_host
 int compass_gemm_rs_sequential_noalloc(const compass_problem* problem, const void* const* A, const void* const* B,
                                        void* const* Out, void* cuda_stream);
 
+/* Bound, in microseconds, of every device-side wait of later launches (default
+ * 2,000,000).  A wait that exceeds it makes the kernel record
+ * COMPASS_ERR_TIMEOUT and return instead of spinning.  0 restores the default. */
+int compass_set_wait_limit_us(uint32_t microseconds);
 const char* compass_status_string(int status);
 int compass_last_cuda_error(void);
 /* Number of kernels this library has launched since it was loaded. */

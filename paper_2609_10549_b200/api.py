@@ -34,6 +34,7 @@ EXPORTS = (
     "compass_calib_fit_decomp", "compass_calib_fit_fusion", "compass_workspace_bytes", "compass_workspace_init",
     "compass_read_status", "compass_launch_plan", "compass_fused_host", "compass_status_string",
     "compass_last_cuda_error", "compass_kernel_launch_count", "compass_gemm_rs_sequential_noalloc",
+    "compass_set_wait_limit_us",
 )
 
 
@@ -100,6 +101,7 @@ def lib() -> C.CDLL:
         L.compass_fused_host.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t),
                                          C.c_void_p, C.c_size_t, C.c_void_p]
         L.compass_gemm_rs_sequential_noalloc.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p]
+        L.compass_set_wait_limit_us.argtypes = [C.c_uint32]
         L.compass_status_string.argtypes = [C.c_int]
         L.compass_status_string.restype = C.c_char_p
         L.compass_last_cuda_error.restype = C.c_int
@@ -114,6 +116,10 @@ def status_string(status: int) -> str:
 
 def last_cuda_error() -> int:
     return int(lib().compass_last_cuda_error())
+
+
+def compass_set_wait_limit_us(microseconds: int) -> None:
+    _check(lib().compass_set_wait_limit_us(int(microseconds)), "compass_set_wait_limit_us")
 
 
 def kernel_launch_count() -> int:

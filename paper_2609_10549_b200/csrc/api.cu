@@ -12,6 +12,7 @@ namespace {
 
 std::atomic<int> g_last_cuda_error{0};
 std::atomic<uint64_t> g_kernel_launches{0};
+std::atomic<uint32_t> g_wait_limit_us{0};
 
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -218,7 +219,6 @@ int fused_call(const compass_problem* pr, int op, const void* const* A, const vo
   if (st != COMPASS_OK) return st;
   st = validate_workspace(pr, COMPASS_WS_FUSED, ws, ws_bytes);
   if (st != COMPASS_OK) return st;
-  if (op == COMPASS_OP_GEMM_RS && pr->rs_variant == COMPASS_RS_RING_RMW) return COMPASS_ERR_UNSUPPORTED;
   static thread_local GemmLaunch L;
   st = plan_fused(pr, &L, nullptr);
   if (st != COMPASS_OK) return st;
@@ -367,6 +367,7 @@ int record_cuda_error(cudaError_t e) {
   return COMPASS_ERR_CUDA;
 }
 void count_kernel_launch() { g_kernel_launches.fetch_add(1, std::memory_order_relaxed); }
+uint32_t default_wait_limit_us() { return g_wait_limit_us.load(std::memory_order_relaxed); }
 
 }  // namespace compass
 
@@ -509,5 +510,9 @@ extern "C" const char* compass_status_string(int status) {
   }
 }
 
+extern "C" int compass_set_wait_limit_us(uint32_t microseconds) {
+  g_wait_limit_us.store(microseconds, std::memory_order_relaxed);
+  return COMPASS_OK;
+}
 extern "C" int compass_last_cuda_error(void) { return g_last_cuda_error.load(); }
 extern "C" uint64_t compass_kernel_launch_count(void) { return g_kernel_launches.load(); }

@@ -9,7 +9,9 @@
 //   AllGather+GEMM: the A tile of a block is TMA-loaded straight from the shard
 //     of the rank that owns the partition (gather by address);
 //   GEMM+ReduceScatter, segmented K: the k-loop of a tile runs over the P ranks'
-//     K slices in ring order into one TMEM accumulator (in-kernel reduction).
+//     K slices in ring order into one TMEM accumulator (in-kernel reduction);
+//   GEMM+ReduceScatter, ring read-modify-write: every rank's partial tile is
+//     added by the epilogue into the owner's rows in ring order.
 //
 // Two modes of the same kernel:
 //   pair   (default when a block has >= 256 rows): a cluster of two CTAs owns a
@@ -99,6 +101,23 @@ __device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, Con
     }
   }
   report_timeout(p, ctl, site, tile);
+  return false;
+}
+
+// Bounded wait until a tile counter in global memory reaches `target`.
+__device__ __forceinline__ bool wait_counter(const int* counter, int target, Control* ctl, const GemmParams& p, int tile) {
+  const uint64_t t0 = globaltimer_ns();
+  const uint64_t limit = uint64_t(p.wait_limit_us) * 1000ull;
+  for (uint32_t spins = 0; spins < (1u << 30); ++spins) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= target) return true;
+    if ((spins & 0x3F) == 0x3F) {
+      if (*reinterpret_cast<volatile int*>(&ctl->abort)) return false;
+      if (globaltimer_ns() - t0 > limit) break;
+    }
+  }
+  report_timeout(p, ctl, WAIT_TILE_COUNTER, tile);
   return false;
 }
 
@@ -290,6 +309,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     }
   } else {
     // ---------------------------------------------------------------- epilogue
+    constexpr int kWarpsPerTile = kPair ? 2 * kEpilogueWarps : kEpilogueWarps;
     const int quarter = warp & 3;               // TMEM lanes this warp may touch
     const int row_in_tile = int(cta_rank) * BM + quarter * 32 + lane;
     uint32_t it = 0;
@@ -306,6 +326,23 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       const int nchunks = (ncols + 31) >> 5;
       __nv_bfloat16* orow = p.out[b.out_idx] + int64_t(b.out_row0 + row_in_block) * p.ldo + int64_t(tc.nt) * BN;
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
+
+      // Ring read-modify-write: contributor `step` of a partition adds its
+      // partial tile to the running sum that contributor step-1 left in the
+      // owner's rows.  One counter per output tile counts the epilogue warps
+      // that have finished; contributor s starts when all warps of s-1 have.
+      const bool rmw = p.epilogue == EPI_RING_RMW;
+      const bool add_previous = rmw && b.step > 0;
+      int* counter = nullptr;
+      if (rmw) {
+        counter = p.tile_counters + (int64_t(b.part) * p.tiles_m + tc.mt) * p.tiles_n + tc.nt;
+        if (add_previous) {
+          int ready = 1;
+          if (lane == 0) ready = wait_counter(counter, int(b.step) * kWarpsPerTile, ctl, p, t) ? 1 : 0;
+          ready = __shfl_sync(0xffffffffu, ready, 0);
+          if (!ready) break;
+        }
+      }
       for (int c = 0; c < nchunks; ++c) {
         uint32_t v[32];
         tmem_ld_32x32b_x32(taddr + c * 32, v);
@@ -323,14 +360,36 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             if (c * 32 + g * 8 < ncols) {
+              uint4* dst = reinterpret_cast<uint4*>(orow + c * 32 + g * 8);
+              float f[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[g * 8 + i]);
+              if (add_previous) {
+                const uint4 old = __ldcg(dst);          // written by another SM: read it from L2
+                const uint32_t w[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  f[2 * i + 0] += __uint_as_float(w[i] << 16);
+                  f[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
+                }
+              }
               uint4 q;
-              q.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
-              q.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
-              q.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
-              q.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
-              *reinterpret_cast<uint4*>(orow + c * 32 + g * 8) = q;
+              q.x = pack_bf16x2(f[0], f[1]);
+              q.y = pack_bf16x2(f[2], f[3]);
+              q.z = pack_bf16x2(f[4], f[5]);
+              q.w = pack_bf16x2(f[6], f[7]);
+              *dst = q;
             }
           }
+        }
+      }
+      if (rmw) {
+        __threadfence();          // this lane's stores are visible device-wide before the counter moves
+        __syncwarp();
+        if (lane == 0) {
+          const int before = atomicAdd(counter, 1);
+          // the last warp of the last contributor leaves the counter at zero for the next call
+          if (int(b.step) == p.last_step && before == (p.last_step + 1) * kWarpsPerTile - 1) atomicExch(counter, 0);
         }
       }
     }
@@ -457,7 +516,7 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   p.total_tiles = L.n_blocks * p.tiles_m * p.tiles_n;
   p.epilogue = L.epilogue;
   p.last_step = L.last_step;
-  p.wait_limit_us = 2000000u;
+  p.wait_limit_us = L.wait_limit_us ? L.wait_limit_us : (default_wait_limit_us() ? default_wait_limit_us() : 2000000u);
   p.a_hint = L.a_hint;
   p.b_hint = L.b_hint;
 

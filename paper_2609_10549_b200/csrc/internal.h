@@ -101,6 +101,7 @@ struct GemmLaunch {
   int epilogue = EPI_STORE;
   int mode = GEMM_MODE_AUTO;
   int a_hint = 0, b_hint = 0;
+  uint32_t wait_limit_us = 0;   // 0 = default bound of the device-side waits
   int last_step = 0;
   int n_blocks = 0;
   BlockDesc blocks[kMaxBlocks];
@@ -121,6 +122,7 @@ int launch_reduce_partials(const void* const* partial, int P, void* const* out, 
 // api.cu
 int record_cuda_error(cudaError_t e);
 void count_kernel_launch();
+uint32_t default_wait_limit_us();   // 0 = built-in default
 
 // schedule.cpp
 int build_schedule(int op, int P, int rings, int64_t M, compass_sched_entry* out);   // out has rings*P*P slots

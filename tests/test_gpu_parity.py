@@ -199,3 +199,77 @@ def test_repeated_calls_give_identical_bits():
     second, _, _ = gu.run_fused(w, A, B)
     for x, y in zip(first, second):
         assert np.array_equal(x, y)
+
+
+# ---- GEMM+ReduceScatter, ring read-modify-write variant --------------------------------------
+
+def check_ring(outs, refs, what, P):
+    """The running sum is rounded to BF16 once per contributor, so the RMS error
+    may reach sqrt(P) roundings of 2^-9 relative each; the per-element
+    acceptance rule is unchanged."""
+    for r, (got, ref) in enumerate(zip(outs, refs)):
+        rep = compare.check(got, ref)
+        assert rep.violations == 0, f"{what} rank {r}: {rep}"
+        assert rep.rms_rel <= 2.0 ** -9 * max(1.0, P ** 0.5), f"{what} rank {r}: {rep}"
+
+
+@pytest.mark.parametrize("P,m,N,K,rings", RS_SHAPES)
+def test_gemm_rs_ring_rmw_small_shapes(P, m, N, K, rings):
+    w = small(wl.OP_GEMM_RS, P, m, N, K, dist=0.05)
+    A, B = wl.make_inputs(w)
+    outs, status, guards = gu.run_fused(w, A, B, rings=rings, rs_variant=api.RS_RING_RMW)
+    assert status == (api.OK, 0) and guards
+    check_ring(outs, ops.gemm_rs(A, B, rings=rings), w.name, P)
+
+
+def test_ring_rmw_integers_exact_and_counters_return_to_zero():
+    w = wl.Workload("ints-ring", wl.OP_GEMM_RS, P=4, M=4 * 512, N=520, K=64)
+    A_bits, B_bits = wl.make_structured_inputs(w, "index")       # every running sum is a small integer: no rounding
+    pr = gu.problem_of(w, rs_variant=api.RS_RING_RMW)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    ws = api.alloc_workspace(pr)
+    ref = ops.gemm_rs(A_bits, B_bits)
+    for _ in range(2):                                           # the second call reuses the counters
+        outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        api.compass_gemm_rs(pr, A, B, [o.view for o in outs], ws)
+        assert api.compass_read_status(ws) == (api.OK, 0)
+        for o, r in zip(outs, ref):
+            assert np.array_equal(ops.bf16_bits_to_f64(o.bits()), r)
+        assert int(ws[api.STATUS_BYTES:].view(torch.int32).abs().sum().item()) == 0
+
+
+def test_config3_ring_rmw_full_size_sampled():
+    w = wl.C3_RS
+    A, B = wl.make_inputs(w)
+    outs, status, guards = gu.run_fused(w, A, B, rs_variant=api.RS_RING_RMW)
+    assert status == (api.OK, 0) and guards
+    rows = gu.sample_rows(w.M, w.P, 2)
+    for c, (local, ref) in ops.gemm_rs_rows(A, B, rows).items():
+        rep = compare.check(outs[c][local], ref)
+        assert rep.violations == 0 and rep.rms_rel <= 2.0 ** -9 * w.P ** 0.5, f"{w.name} chunk {c}: {rep}"
+
+
+def test_bounded_wait_reports_timeout_and_the_context_survives():
+    """A tile counter that no contributor will ever raise (the host plants a
+    negative value) makes the ring epilogue's wait run out: the kernel must
+    return with COMPASS_ERR_TIMEOUT in the status block, and the next call on
+    a re-initialised workspace must work."""
+    w = small(wl.OP_GEMM_RS, 2, 256, 256, 64, dist=0.05)
+    A_bits, B_bits = wl.make_inputs(w)
+    pr = gu.problem_of(w, rs_variant=api.RS_RING_RMW)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    ws = api.alloc_workspace(pr)
+    ws[api.STATUS_BYTES:].view(torch.int32).fill_(-1000)
+    api.compass_set_wait_limit_us(20000)
+    try:
+        api.compass_gemm_rs(pr, A, B, [o.view for o in outs], ws)
+        status, detail = api.compass_read_status(ws)
+    finally:
+        api.compass_set_wait_limit_us(0)
+    assert status == api.ERR_TIMEOUT and detail in (3, 4, 6)      # a tile-counter wait or a wait behind it
+    torch.cuda.synchronize()
+    api.compass_workspace_init(ws)
+    api.compass_gemm_rs(pr, A, B, [o.view for o in outs], ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    check_ring([o.bits() for o in outs], ops.gemm_rs(A_bits, B_bits), w.name, w.P)
