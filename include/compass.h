@@ -213,6 +213,9 @@ int compass_model_fusion_time(double t_comp, double t_comm, int n_chunks, double
  * (t_comp[i], t_comm[i], d[i] > 1, t_measured[i]) regressed on d. */
 int compass_calib_fit_decomp(const double* t_comp, const double* t_comm, const int* d, const double* t_measured,
                              size_t n, double* alpha, double* beta);
+/* Least-squares line y = a + b*x (the linear T_comp and T_comm models of
+ * Section IV-B are fitted with it); a single distinct x gives (mean y, 0). */
+int compass_calib_fit_line(const double* x, const double* y, size_t n, double* a, double* b);
 /* Residual of Eq. 7 per synchronisation point regressed on the message volume m. */
 int compass_calib_fit_fusion(const double* t_comp, const double* t_comm, const int* n_chunks, const double* m_volume,
                              const double* t_measured, size_t n, double* alpha_f, double* beta_f);

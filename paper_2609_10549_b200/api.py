@@ -34,7 +34,7 @@ EXPORTS = (
     "compass_calib_fit_decomp", "compass_calib_fit_fusion", "compass_workspace_bytes", "compass_workspace_init",
     "compass_read_status", "compass_launch_plan", "compass_fused_host", "compass_status_string",
     "compass_last_cuda_error", "compass_kernel_launch_count", "compass_gemm_rs_sequential_noalloc",
-    "compass_set_wait_limit_us",
+    "compass_set_wait_limit_us", "compass_calib_fit_line",
 )
 
 
@@ -94,6 +94,7 @@ def lib() -> C.CDLL:
         dp, ip = C.POINTER(C.c_double), C.POINTER(C.c_int)
         L.compass_calib_fit_decomp.argtypes = [dp, dp, ip, dp, C.c_size_t, dp, dp]
         L.compass_calib_fit_fusion.argtypes = [dp, dp, ip, dp, dp, C.c_size_t, dp, dp]
+        L.compass_calib_fit_line.argtypes = [dp, dp, C.c_size_t, dp, dp]
         L.compass_workspace_bytes.argtypes = [C.POINTER(Problem), C.c_int, C.POINTER(C.c_size_t)]
         L.compass_workspace_init.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
         L.compass_read_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]
@@ -188,6 +189,12 @@ def compass_calib_fit_decomp(t_comp, t_comm, d, t_measured):
     a, b = C.c_double(), C.c_double()
     _check(lib().compass_calib_fit_decomp(_darr(t_comp), _darr(t_comm), _iarr(d), _darr(t_measured), len(d),
                                           C.byref(a), C.byref(b)), "compass_calib_fit_decomp")
+    return a.value, b.value
+
+
+def compass_calib_fit_line(x, y):
+    a, b = C.c_double(), C.c_double()
+    _check(lib().compass_calib_fit_line(_darr(x), _darr(y), len(x), C.byref(a), C.byref(b)), "compass_calib_fit_line")
     return a.value, b.value
 
 

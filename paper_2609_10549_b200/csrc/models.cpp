@@ -161,6 +161,11 @@ extern "C" int compass_calib_fit_decomp(const double* t_comp, const double* t_co
   return ols(xs, ys, n, alpha, beta) ? COMPASS_OK : COMPASS_ERR_INVALID_ARG;
 }
 
+extern "C" int compass_calib_fit_line(const double* x, const double* y, size_t n, double* a, double* b) {
+  if (!x || !y || !a || !b || n == 0) return COMPASS_ERR_INVALID_ARG;
+  return ols(x, y, n, a, b) ? COMPASS_OK : COMPASS_ERR_INVALID_ARG;
+}
+
 extern "C" int compass_calib_fit_fusion(const double* t_comp, const double* t_comm, const int* n_chunks,
                                         const double* m_volume, const double* t_meas, size_t n, double* alpha_f,
                                         double* beta_f) {

@@ -137,6 +137,9 @@ def test_calibration_matches_oracle():
     n = [4, 8, 4, 8]; vol = [1e6, 4e6, 2e6, 8e6]; c4 = [100.0, 30.0, 55.0, 70.0]; m4 = [40.0, 90.0, 55.0, 10.0]
     tf = [omo.fusion_time(c, m, nn, 3.0, 2e-6, v) * (1 + 0.01 * rng.standard_normal())
           for c, m, nn, v in zip(c4, m4, n, vol)]
+    assert api.compass_calib_fit_line([1.0, 2.0, 4.0], [3.5, 5.0, 8.0]) == (pytest.approx(omo.ols([1.0, 2.0, 4.0], [3.5, 5.0, 8.0])[0]),
+                                                                            pytest.approx(omo.ols([1.0, 2.0, 4.0], [3.5, 5.0, 8.0])[1]))
+    assert api.compass_calib_fit_line([2.0, 2.0], [1.0, 3.0]) == (2.0, 0.0)
     a_lib, b_lib = api.compass_calib_fit_fusion(c4, m4, n, vol, tf)
     a_ref, b_ref = omo.fit_fusion_overhead(list(zip(c4, m4, n, vol, tf)))
     assert a_lib == pytest.approx(a_ref, rel=1e-9) and b_lib == pytest.approx(b_ref, rel=1e-9)
