@@ -36,9 +36,9 @@ UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes per launch of the GEMM kernel from the ncu capture summarised in
-# profiles/ (null until a capture exists): {"C2": bytes, "C3": bytes}.
-NCU_TRAFFIC_BYTES = None
+# DRAM bytes (read + written) per launch of the GEMM kernel from the ncu capture summarised in
+# profiles/gemm_kernel_pair_k128_C2_C3.md.
+NCU_TRAFFIC_BYTES = {"C2": 316.6e6, "C3": 1024.0e6}
 
 
 def env_int(name, default):
@@ -326,6 +326,24 @@ def interdecom_report(torch, api):
 
 
 # ---------------------------------------------------------------------------------
+# aggregation over replicas (one process per GPU; every rank runs the same workload on its own GPU)
+
+def reduce_over_ranks(dist, timings_ms, launches, device):
+    """Device timings: max over ranks; kernel launches: sum over ranks."""
+    import torch
+    t = torch.tensor(list(timings_ms), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    n = torch.tensor([int(launches)], dtype=torch.int64, device=device)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t.tolist()], int(n.item())
+
+
+def aggregate_tflops(world, flops_per_replica_step, ms_per_step):
+    """Whole-job throughput: all replicas' FLOPs over the slowest replica's time."""
+    return world * flops_per_replica_step / (ms_per_step * 1e-3) / 1e12
+
+
+# ---------------------------------------------------------------------------------
 # our arm
 
 def run_ours(args, w_ag, w_rs):
@@ -440,17 +458,12 @@ def run_ours(args, w_ag, w_rs):
 
     # max over ranks
     if world > 1:
-        t = torch.tensor([total_ms, e2e_ms, t_ag, t_rs], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms, t_ag, t_rs = [float(x) for x in t.tolist()]
-        lt = torch.tensor([launches], dtype=torch.int64, device="cuda")
-        dist.all_reduce(lt, op=dist.ReduceOp.SUM)
-        launches = int(lt.item())
+        (total_ms, e2e_ms, t_ag, t_rs), launches = reduce_over_ranks(dist, [total_ms, e2e_ms, t_ag, t_rs], launches, "cuda")
 
     if rank == 0:
         flops_step = w_ag.flops + w_rs.flops
         ms_per_step = total_ms / args.steps
-        value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+        value = aggregate_tflops(world, flops_step, ms_per_step)
         peaks, peak_src = measured_peaks()
         kernel_s = (t_ag + t_rs) * 1e-3 / 2.0            # average duration of one launch of the GEMM kernel
         achieved = (flops_step / 2.0) / kernel_s / 1e12

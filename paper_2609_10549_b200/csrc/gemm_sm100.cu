@@ -134,6 +134,36 @@ __device__ __forceinline__ TileCoord decode_tile(const GemmParams& p, int t) {
   return c;
 }
 
+// Walks the sequence of k-stages one work unit loads: for every tile of the
+// unit (t, t + n_units, ...), every K segment, every k-stage of the segment.
+template <bool kPair>
+struct StageIter {
+  int t, step, cta_rank;
+  int seg, kb;
+  int am, bm, a_row, b_row;
+  __device__ StageIter(const GemmParams& p, int unit, int n_units, int rank) : t(unit), step(n_units), cta_rank(rank), seg(0), kb(0) {
+    if (valid(p)) enter(p);
+  }
+  __device__ bool valid(const GemmParams& p) const { return t < p.total_tiles; }
+  __device__ void enter(const GemmParams& p) {      // refresh what depends on (t, seg)
+    const TileCoord tc = decode_tile(p, t);
+    const BlockDesc& b = p.blocks[tc.blk];
+    a_row = b.a_row0 + tc.mt * Cfg<kPair>::kTileRows + cta_rank * BM;
+    b_row = tc.nt * BN + cta_rank * Cfg<kPair>::kBRows;
+    am = (p.n_seg > 1) ? p.seg_rank[tc.blk][seg] : b.a_map;
+    bm = (p.n_seg > 1) ? am : b.b_map;
+  }
+  __device__ void next(const GemmParams& p) {
+    if (++kb < p.kb_per_seg) return;
+    kb = 0;
+    if (++seg == p.n_seg) {
+      seg = 0;
+      t += step;
+    }
+    if (valid(p)) enter(p);
+  }
+};
+
 template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
   using C = Cfg<kPair>;
@@ -192,50 +222,53 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       int stage = 0;
       uint32_t phase = 0;
       uint32_t issued = 0;
-      bool ok = true;
       const uint64_t pol_a = make_l2_policy(p.a_hint);
       const uint64_t pol_b = make_l2_policy(p.b_hint);
-      for (int t = unit; ok && t < p.total_tiles; t += n_units) {
-        const TileCoord tc = decode_tile(p, t);
-        const BlockDesc& b = p.blocks[tc.blk];
-        const int a_row = b.a_row0 + tc.mt * C::kTileRows + int(cta_rank) * BM;
-        const int b_row = tc.nt * BN + int(cta_rank) * C::kBRows;
-        for (int seg = 0; ok && seg < p.n_seg; ++seg) {
-          const int am = (p.n_seg > 1) ? p.seg_rank[tc.blk][seg] : b.a_map;
-          const int bm = (p.n_seg > 1) ? am : b.b_map;
-          for (int kb = 0; kb < p.kb_per_seg; ++kb) {
-            if (!wait_bounded(&ctl->empty[stage], phase ^ 1u, ctl, p, WAIT_SMEM_EMPTY, t)) {
-              ok = false;
-              break;
-            }
-            const int kx = kb * C::kStageK;
-            if (kPair) {
-              // both CTAs' loads complete on the leader's barrier, which expects the bytes of both
-              const uint32_t full_addr = map_to_cta(smem_u32(&ctl->full[stage]), 0);
-              if (leader) mbar_arrive_expect_tx(&ctl->full[stage], C::kFullTxBytes);
+      // `ld` walks this unit's (tile, segment, k-stage) sequence; `pf` can run
+      // p.prefetch_stages ahead of it and pull the boxes into L2 only.  Off by
+      // default: on B200 the prefetches compete with the loads for the same
+      // request path and slow the kernel down (measured: up to 2x).
+      StageIter<kPair> ld(p, unit, n_units, int(cta_rank));
+      StageIter<kPair> pf(p, unit, n_units, int(cta_rank));
+      for (int i = 0; i < p.prefetch_stages && pf.valid(p); ++i) pf.next(p);
+      while (ld.valid(p)) {
+        if (!wait_bounded(&ctl->empty[stage], phase ^ 1u, ctl, p, WAIT_SMEM_EMPTY, ld.t)) break;
+        const int kx = ld.kb * C::kStageK;
+        if (kPair) {
+          // both CTAs' loads complete on the leader's barrier, which expects the bytes of both
+          const uint32_t full_addr = map_to_cta(smem_u32(&ctl->full[stage]), 0);
+          if (leader) mbar_arrive_expect_tx(&ctl->full[stage], C::kFullTxBytes);
 #pragma unroll
-              for (int at = 0; at < C::kAtoms; ++at) {
-                tma_load_2d_pair_hint(smem_a + stage * C::kATileBytes + at * C::kAAtomBytes, &p.a_maps[am], full_addr,
-                                      kx + at * BK, a_row, pol_a);
-                tma_load_2d_pair_hint(smem_b + stage * C::kBTileBytes + at * C::kBAtomBytes, &p.b_maps[bm], full_addr,
-                                      kx + at * BK, b_row, pol_b);
-              }
-            } else {
-              mbar_arrive_expect_tx(&ctl->full[stage], C::kFullTxBytes);
-#pragma unroll
-              for (int at = 0; at < C::kAtoms; ++at) {
-                tma_load_2d_hint(smem_a + stage * C::kATileBytes + at * C::kAAtomBytes, &p.a_maps[am], &ctl->full[stage],
-                                 kx + at * BK, a_row, pol_a);
-                tma_load_2d_hint(smem_b + stage * C::kBTileBytes + at * C::kBAtomBytes, &p.b_maps[bm], &ctl->full[stage],
-                                 kx + at * BK, b_row, pol_b);
-              }
-            }
-            ++issued;
-            if (++stage == C::kStages) {
-              stage = 0;
-              phase ^= 1u;
-            }
+          for (int at = 0; at < C::kAtoms; ++at) {
+            tma_load_2d_pair_hint(smem_a + stage * C::kATileBytes + at * C::kAAtomBytes, &p.a_maps[ld.am], full_addr,
+                                  kx + at * BK, ld.a_row, pol_a);
+            tma_load_2d_pair_hint(smem_b + stage * C::kBTileBytes + at * C::kBAtomBytes, &p.b_maps[ld.bm], full_addr,
+                                  kx + at * BK, ld.b_row, pol_b);
           }
+        } else {
+          mbar_arrive_expect_tx(&ctl->full[stage], C::kFullTxBytes);
+#pragma unroll
+          for (int at = 0; at < C::kAtoms; ++at) {
+            tma_load_2d_hint(smem_a + stage * C::kATileBytes + at * C::kAAtomBytes, &p.a_maps[ld.am], &ctl->full[stage],
+                             kx + at * BK, ld.a_row, pol_a);
+            tma_load_2d_hint(smem_b + stage * C::kBTileBytes + at * C::kBAtomBytes, &p.b_maps[ld.bm], &ctl->full[stage],
+                             kx + at * BK, ld.b_row, pol_b);
+          }
+        }
+        if (p.prefetch_stages > 0 && pf.valid(p)) {
+          const int px = pf.kb * C::kStageK;
+#pragma unroll
+          for (int at = 0; at < C::kAtoms; ++at) {
+            tma_prefetch_l2_2d(&p.a_maps[pf.am], px + at * BK, pf.a_row);
+            tma_prefetch_l2_2d(&p.b_maps[pf.bm], px + at * BK, pf.b_row);
+          }
+          pf.next(p);
+        }
+        ld.next(p);
+        ++issued;
+        if (++stage == C::kStages) {
+          stage = 0;
+          phase ^= 1u;
         }
       }
       // Do not leave the CTA while bulk copies may still be writing shared
@@ -254,8 +287,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
-    if (lane == 0 && leader) {
+    // The whole warp walks the loop so that addresses and descriptors are
+    // warp-uniform values; only the issue instructions are executed by one lane.
+    if (leader) {
       constexpr uint32_t idesc = umma_idesc_bf16_f32(kPair ? 2 * BM : BM, BN);
+      constexpr int kFullSteps = C::kStageK / UMMA_K;
+      const bool issuer = lane == 0;
+      const uint64_t desc_a0 = umma_smem_desc_sw128(smem_u32(smem_a));
+      const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(smem_b));
       int stage = 0;
       uint32_t phase = 0;
       uint32_t it = 0;
@@ -263,49 +302,67 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       for (int t = unit; ok && t < p.total_tiles; t += n_units, ++it) {
         const uint32_t buf = it & 1u;
         const uint32_t acc_phase = (it >> 1) & 1u;
-        if (!wait_bounded(&ctl->acc_empty[buf], acc_phase ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
+        ok = __all_sync(0xffffffffu, wait_bounded(&ctl->acc_empty[buf], acc_phase ^ 1u, ctl, p, WAIT_ACC_EMPTY, t));
+        if (!ok) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + buf * BN;
         int kb_in_seg = 0;
         for (int kb = 0; kb < total_kb; ++kb) {
-          if (!wait_bounded(&ctl->full[stage], phase, ctl, p, WAIT_SMEM_FULL, t)) {
-            ok = false;
-            break;
-          }
+          ok = __all_sync(0xffffffffu, wait_bounded(&ctl->full[stage], phase, ctl, p, WAIT_SMEM_FULL, t));
+          if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t a_base = smem_u32(smem_a + stage * C::kATileBytes);
-          const uint32_t b_base = smem_u32(smem_b + stage * C::kBTileBytes);
-          const int ksteps = (kb_in_seg == p.kb_per_seg - 1) ? p.tail_ksteps : C::kStageK / UMMA_K;
-          for (int ks = 0; ks < ksteps; ++ks) {
-            // a 64-element atom holds 4 steps of 16 elements = 32 bytes each: +2 in the descriptor's address field
-            const int at = ks >> 2, k = ks & 3;
-            const uint64_t da = umma_smem_desc_sw128(a_base + at * C::kAAtomBytes) + uint64_t(k * 2);
-            const uint64_t db = umma_smem_desc_sw128(b_base + at * C::kBAtomBytes) + uint64_t(k * 2);
-            const uint32_t acc = (kb | ks) != 0 ? 1u : 0u;
-            if (kPair) umma_bf16_pair(d_tmem, da, db, idesc, acc);
-            else umma_bf16(d_tmem, da, db, idesc, acc);
+          // descriptor address fields count 16-byte units
+          const uint64_t da = desc_a0 + uint64_t((stage * C::kATileBytes) >> 4);
+          const uint64_t db = desc_b0 + uint64_t((stage * C::kBTileBytes) >> 4);
+          const bool last_of_seg = kb_in_seg == p.kb_per_seg - 1;
+          if (!last_of_seg || p.tail_ksteps == kFullSteps) {
+#pragma unroll
+            for (int ks = 0; ks < kFullSteps; ++ks) {
+              // a 64-element atom holds 4 steps of 16 elements = 32 bytes each: +2 in the address field
+              const uint64_t a_k = da + uint64_t(((ks >> 2) * C::kAAtomBytes >> 4) + (ks & 3) * 2);
+              const uint64_t b_k = db + uint64_t(((ks >> 2) * C::kBAtomBytes >> 4) + (ks & 3) * 2);
+              const uint32_t acc = (kb | ks) != 0 ? 1u : 0u;
+              if (issuer) {
+                if (kPair) umma_bf16_pair(d_tmem, a_k, b_k, idesc, acc);
+                else umma_bf16(d_tmem, a_k, b_k, idesc, acc);
+              }
+            }
+          } else {
+            for (int ks = 0; ks < p.tail_ksteps; ++ks) {
+              const uint64_t a_k = da + uint64_t(((ks >> 2) * C::kAAtomBytes >> 4) + (ks & 3) * 2);
+              const uint64_t b_k = db + uint64_t(((ks >> 2) * C::kBAtomBytes >> 4) + (ks & 3) * 2);
+              const uint32_t acc = (kb | ks) != 0 ? 1u : 0u;
+              if (issuer) {
+                if (kPair) umma_bf16_pair(d_tmem, a_k, b_k, idesc, acc);
+                else umma_bf16(d_tmem, a_k, b_k, idesc, acc);
+              }
+            }
           }
           // the stage is reusable (in both CTAs) once these MMAs have read it
-          if (kPair) umma_commit_pair(&ctl->empty[stage], 0x3);
-          else umma_commit(&ctl->empty[stage]);
+          if (issuer) {
+            if (kPair) umma_commit_pair(&ctl->empty[stage], 0x3);
+            else umma_commit(&ctl->empty[stage]);
+          }
           if (++kb_in_seg == p.kb_per_seg) kb_in_seg = 0;
           if (++stage == C::kStages) {
             stage = 0;
             phase ^= 1u;
           }
         }
-        if (ok) {   // accumulator complete: wake the epilogue (of both CTAs)
+        if (ok && issuer) {   // accumulator complete: wake the epilogue (of both CTAs)
           if (kPair) umma_commit_pair(&ctl->acc_full[buf], 0x3);
           else umma_commit(&ctl->acc_full[buf]);
         }
+        __syncwarp();
       }
-      if (*reinterpret_cast<volatile int*>(&ctl->abort)) {
+      if (issuer && *reinterpret_cast<volatile int*>(&ctl->abort)) {
         // Gave up somewhere: wait for whatever the tensor core still has in
         // flight before tensor memory is released.
         if (kPair) umma_commit_pair(&ctl->drain, 0x1);
         else umma_commit(&ctl->drain);
         wait_bounded(&ctl->drain, 0, ctl, p, WAIT_DRAIN, -2);
       }
+      __syncwarp();
     }
   } else {
     // ---------------------------------------------------------------- epilogue
@@ -517,6 +574,7 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   p.epilogue = L.epilogue;
   p.last_step = L.last_step;
   p.wait_limit_us = L.wait_limit_us ? L.wait_limit_us : (default_wait_limit_us() ? default_wait_limit_us() : 2000000u);
+  p.prefetch_stages = L.prefetch_stages;
   p.a_hint = L.a_hint;
   p.b_hint = L.b_hint;
 

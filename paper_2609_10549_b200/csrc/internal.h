@@ -80,6 +80,7 @@ struct GemmParams {
   int32_t last_step;       // ring RMW: step index of the final contributor (P-1)
   uint32_t wait_limit_us;  // bound of every device-side wait
   int32_t a_hint, b_hint;  // L2 eviction priority of the A / B tile loads (ptx::L2Hint)
+  int32_t prefetch_stages; // how many k-stages ahead of the shared-memory loads operands are prefetched into L2 (0 = off)
   StatusBlock* status;
   int32_t* tile_counters;  // ring RMW only
   uint8_t seg_rank[kMaxSegBlocks][kMaxP];   // segmented-K: tensor index of segment s of block b
@@ -101,6 +102,7 @@ struct GemmLaunch {
   int epilogue = EPI_STORE;
   int mode = GEMM_MODE_AUTO;
   int a_hint = 0, b_hint = 0;
+  int prefetch_stages = 0;
   uint32_t wait_limit_us = 0;   // 0 = default bound of the device-side waits
   int last_step = 0;
   int n_blocks = 0;
