@@ -99,7 +99,6 @@ extern "C" int compass_gemm_rs_sequential_noalloc(const compass_problem* pr, con
   L.rows_per_block = int(m);
   L.epilogue = EPI_STORE;
   L.mode = GEMM_MODE_AUTO;
-  L.a_hint = L.b_hint = 0;
   L.status = reinterpret_cast<StatusBlock*>(scratch);
   L.tile_counters = nullptr;
   int n = 0;
