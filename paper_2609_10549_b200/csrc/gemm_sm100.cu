@@ -287,12 +287,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
-    // The whole warp walks the loop so that addresses and descriptors are
-    // warp-uniform values; only the issue instructions are executed by one lane.
-    if (leader) {
+    // One lane runs the whole loop (a per-instruction "if (lane == 0)" inside a
+    // 32-lane loop costs a divergence per MMA and slows the issue stream).
+    if (leader && lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16_f32(kPair ? 2 * BM : BM, BN);
       constexpr int kFullSteps = C::kStageK / UMMA_K;
-      const bool issuer = lane == 0;
       const uint64_t desc_a0 = umma_smem_desc_sw128(smem_u32(smem_a));
       const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(smem_b));
       int stage = 0;
@@ -302,67 +301,58 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       for (int t = unit; ok && t < p.total_tiles; t += n_units, ++it) {
         const uint32_t buf = it & 1u;
         const uint32_t acc_phase = (it >> 1) & 1u;
-        ok = __all_sync(0xffffffffu, wait_bounded(&ctl->acc_empty[buf], acc_phase ^ 1u, ctl, p, WAIT_ACC_EMPTY, t));
-        if (!ok) break;
+        if (!wait_bounded(&ctl->acc_empty[buf], acc_phase ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + buf * BN;
         int kb_in_seg = 0;
         for (int kb = 0; kb < total_kb; ++kb) {
-          ok = __all_sync(0xffffffffu, wait_bounded(&ctl->full[stage], phase, ctl, p, WAIT_SMEM_FULL, t));
-          if (!ok) break;
+          if (!wait_bounded(&ctl->full[stage], phase, ctl, p, WAIT_SMEM_FULL, t)) {
+            ok = false;
+            break;
+          }
           tc_fence_after_sync();
           // descriptor address fields count 16-byte units
           const uint64_t da = desc_a0 + uint64_t((stage * C::kATileBytes) >> 4);
           const uint64_t db = desc_b0 + uint64_t((stage * C::kBTileBytes) >> 4);
-          const bool last_of_seg = kb_in_seg == p.kb_per_seg - 1;
-          if (!last_of_seg || p.tail_ksteps == kFullSteps) {
+          const uint32_t first = kb != 0 ? 1u : 0u;
+          if (kb_in_seg != p.kb_per_seg - 1 || p.tail_ksteps == kFullSteps) {
 #pragma unroll
             for (int ks = 0; ks < kFullSteps; ++ks) {
               // a 64-element atom holds 4 steps of 16 elements = 32 bytes each: +2 in the address field
               const uint64_t a_k = da + uint64_t(((ks >> 2) * C::kAAtomBytes >> 4) + (ks & 3) * 2);
               const uint64_t b_k = db + uint64_t(((ks >> 2) * C::kBAtomBytes >> 4) + (ks & 3) * 2);
-              const uint32_t acc = (kb | ks) != 0 ? 1u : 0u;
-              if (issuer) {
-                if (kPair) umma_bf16_pair(d_tmem, a_k, b_k, idesc, acc);
-                else umma_bf16(d_tmem, a_k, b_k, idesc, acc);
-              }
+              if (kPair) umma_bf16_pair(d_tmem, a_k, b_k, idesc, ks ? 1u : first);
+              else umma_bf16(d_tmem, a_k, b_k, idesc, ks ? 1u : first);
             }
           } else {
             for (int ks = 0; ks < p.tail_ksteps; ++ks) {
               const uint64_t a_k = da + uint64_t(((ks >> 2) * C::kAAtomBytes >> 4) + (ks & 3) * 2);
               const uint64_t b_k = db + uint64_t(((ks >> 2) * C::kBAtomBytes >> 4) + (ks & 3) * 2);
-              const uint32_t acc = (kb | ks) != 0 ? 1u : 0u;
-              if (issuer) {
-                if (kPair) umma_bf16_pair(d_tmem, a_k, b_k, idesc, acc);
-                else umma_bf16(d_tmem, a_k, b_k, idesc, acc);
-              }
+              if (kPair) umma_bf16_pair(d_tmem, a_k, b_k, idesc, ks ? 1u : first);
+              else umma_bf16(d_tmem, a_k, b_k, idesc, ks ? 1u : first);
             }
           }
           // the stage is reusable (in both CTAs) once these MMAs have read it
-          if (issuer) {
-            if (kPair) umma_commit_pair(&ctl->empty[stage], 0x3);
-            else umma_commit(&ctl->empty[stage]);
-          }
+          if (kPair) umma_commit_pair(&ctl->empty[stage], 0x3);
+          else umma_commit(&ctl->empty[stage]);
           if (++kb_in_seg == p.kb_per_seg) kb_in_seg = 0;
           if (++stage == C::kStages) {
             stage = 0;
             phase ^= 1u;
           }
         }
-        if (ok && issuer) {   // accumulator complete: wake the epilogue (of both CTAs)
+        if (ok) {   // accumulator complete: wake the epilogue (of both CTAs)
           if (kPair) umma_commit_pair(&ctl->acc_full[buf], 0x3);
           else umma_commit(&ctl->acc_full[buf]);
         }
-        __syncwarp();
       }
-      if (issuer && *reinterpret_cast<volatile int*>(&ctl->abort)) {
+      if (*reinterpret_cast<volatile int*>(&ctl->abort)) {
         // Gave up somewhere: wait for whatever the tensor core still has in
         // flight before tensor memory is released.
         if (kPair) umma_commit_pair(&ctl->drain, 0x1);
         else umma_commit(&ctl->drain);
         wait_bounded(&ctl->drain, 0, ctl, p, WAIT_DRAIN, -2);
       }
-      __syncwarp();
     }
   } else {
     // ---------------------------------------------------------------- epilogue
@@ -466,6 +456,394 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
   }
 }
 
+// ---- mixed-tile pair kernel ---------------------------------------------------------
+//
+// Same roles and protocol as gemm_kernel<true>, but a launch holds two kinds of
+// tiles, both computed by a pair of CTAs:
+//   big   512 x 256: each CTA owns 256 rows as two 128-row accumulators (TMEM
+//         columns 0..255 and 256..511) that share one B tile.  A k-stage is one
+//         64-wide atom: A block 0, A block 1, B = 3 chunks of 16 KB per CTA,
+//         8 MMAs.  Per 128x256x64 MMA block the CTA loads 24 KB instead of 32.
+//   small 256 x 256: one accumulator, k-stage = two 64-wide atoms (A0, A1, B0,
+//         B1 = 4 chunks), 8 MMAs; accumulators alternate so the epilogue overlaps.
+// Big tiles come first and fill whole waves (their number is a multiple of the
+// number of pairs); the remaining rows are cut into small tiles so that the last,
+// partly filled wave costs half as much.  Shared memory is one FIFO ring of 12
+// chunks; stage j uses barrier slot j & 3 with parity (j >> 2) & 1, and the
+// producer fills stage j once stage j - depth has been released (depth 4 for big,
+// 3 for small stages), which also holds across the change of kind.
+constexpr int kChunkBytes = BM * BK * 2;      // 16 KB: one 128-row, 64-column BF16 box
+constexpr int kChunks = 12;
+constexpr int kSlots = 4;
+
+struct MixedControl {
+  uint64_t full[kSlots];
+  uint64_t empty[kSlots];
+  uint64_t acc_full[2];
+  uint64_t acc_empty[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort;
+};
+// epilogue staging: per epilogue warp 32 rows x 64 BF16 columns, rows padded by 16 bytes (conflict-free 16-byte accesses)
+constexpr int kStageRowBytes = 64 * 2 + 16;
+constexpr int kStageWarpBytes = 32 * kStageRowBytes;
+constexpr size_t kMixedSmemBytes =
+    1024 + size_t(kChunks) * kChunkBytes + sizeof(MixedControl) + 16 + size_t(kEpilogueWarps) * kStageWarpBytes;
+
+struct MixedTile {
+  int big;        // 1 = 512x256, 0 = 256x256
+  int blk, nt;
+  int row0;       // first row of the pair's tile inside the block
+  int valid;
+};
+__device__ __forceinline__ MixedTile decode_mixed(const GemmParams& p, int t) {
+  MixedTile m;
+  int tb;
+  int half = 0;
+  if (t < p.n_big) {
+    m.big = 1;
+    tb = t;
+  } else {
+    m.big = 0;
+    const int u = t - p.n_big;
+    tb = p.n_big + (u >> 1);
+    half = u & 1;
+  }
+  const int per_block = p.big_tiles_m * p.tiles_n;
+  m.blk = tb / per_block;
+  const int w = tb - m.blk * per_block;
+  const int mtb = w / p.tiles_n;
+  m.nt = w - mtb * p.tiles_n;
+  m.row0 = mtb * (4 * BM) + half * (2 * BM);
+  m.valid = m.row0 < p.rows_per_block;
+  return m;
+}
+
+// Walks the k-stages of one pair's tiles: tile, K segment, k-stage.
+struct MixedIter {
+  int t, step, cta_rank;
+  int seg, kb, n_kb;
+  MixedTile tile;
+  int am, bm, a_row, b_row;
+  __device__ MixedIter(const GemmParams& p, int unit, int n_units, int rank) : t(unit), step(n_units), cta_rank(rank), seg(0), kb(0) {
+    skip_invalid(p);
+  }
+  __device__ bool valid(const GemmParams& p) const { return t < p.total_tiles; }
+  __device__ void skip_invalid(const GemmParams& p) {
+    while (t < p.total_tiles) {
+      tile = decode_mixed(p, t);
+      if (tile.valid) {
+        enter(p);
+        return;
+      }
+      t += step;
+    }
+  }
+  __device__ void enter(const GemmParams& p) {
+    const BlockDesc& b = p.blocks[tile.blk];
+    a_row = b.a_row0 + tile.row0 + cta_rank * (tile.big ? 2 * BM : BM);
+    b_row = tile.nt * BN + cta_rank * (BN / 2);
+    am = (p.n_seg > 1) ? p.seg_rank[tile.blk][seg] : b.a_map;
+    bm = (p.n_seg > 1) ? am : b.b_map;
+    n_kb = tile.big ? p.kb_big : p.kb_per_seg;
+  }
+  __device__ void next(const GemmParams& p) {
+    if (++kb < n_kb) return;
+    kb = 0;
+    if (++seg == p.n_seg) {
+      seg = 0;
+      t += step;
+      skip_invalid(p);
+      return;
+    }
+    enter(p);
+  }
+};
+
+__device__ __forceinline__ void report_timeout_m(const GemmParams& p, MixedControl* ctl, int site, int tile) {
+  *reinterpret_cast<volatile int*>(&ctl->abort) = 1;
+  if (atomicCAS(&p.status->code, 0, int(COMPASS_ERR_TIMEOUT)) == 0) {
+    p.status->detail = site;
+    p.status->block_idx = int(blockIdx.x);
+    p.status->tile = tile;
+  }
+}
+__device__ __forceinline__ bool wait_bounded_m(uint64_t* bar, uint32_t parity, MixedControl* ctl, const GemmParams& p, int site,
+                                               int tile) {
+  if (mbar_test_wait(bar, parity)) return true;
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = globaltimer_ns();
+  const uint64_t limit = uint64_t(p.wait_limit_us) * 1000ull;
+  for (uint32_t spins = 1; spins < (1u << 30); ++spins) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spins & 0xFF) == 0) {
+      if (*reinterpret_cast<volatile int*>(&ctl->abort)) return false;
+      if (globaltimer_ns() - t0 > limit) break;
+    }
+  }
+  report_timeout_m(p, ctl, site, tile);
+  return false;
+}
+
+__global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  uint8_t* smem = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
+  MixedControl* ctl = reinterpret_cast<MixedControl*>(smem + kChunks * kChunkBytes);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t cta_rank = cluster_ctarank();
+  const bool leader = cta_rank == 0;
+  const int unit = int(blockIdx.x >> 1);
+  const int n_units = int(gridDim.x >> 1);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kSlots; ++s) {
+      mbar_init(&ctl->full[s], 1);
+      mbar_init(&ctl->empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&ctl->acc_full[b], 1);
+      mbar_init(&ctl->acc_empty[b], 2 * kEpilogueWarps);
+    }
+    mbar_init(&ctl->drain, 1);
+    ctl->abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(&ctl->tmem_base, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = ctl->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      const uint64_t pol_a = make_l2_policy(p.a_hint);
+      const uint64_t pol_b = make_l2_policy(p.b_hint);
+      uint32_t j = 0;          // global stage counter
+      int chunk = 0;           // ring cursor
+      for (MixedIter it(p, unit, n_units, int(cta_rank)); it.valid(p); it.next(p), ++j) {
+        const int big = it.tile.big;
+        const uint32_t depth = big ? 4u : 3u;
+        if (j >= depth) {
+          const uint32_t r = j - depth;      // this stage's chunks are free once stage r has been released
+          if (!wait_bounded_m(&ctl->empty[r & 3u], (r >> 2) & 1u, ctl, p, WAIT_SMEM_EMPTY, it.t)) break;
+        }
+        const uint32_t slot = j & 3u;
+        const uint32_t full_addr = map_to_cta(smem_u32(&ctl->full[slot]), 0);
+        const int nchunks = big ? 3 : 4;
+        if (leader) mbar_arrive_expect_tx(&ctl->full[slot], uint32_t(2 * nchunks * kChunkBytes));
+        uint8_t* c0 = smem + ((chunk + 0) % kChunks) * kChunkBytes;
+        uint8_t* c1 = smem + ((chunk + 1) % kChunks) * kChunkBytes;
+        uint8_t* c2 = smem + ((chunk + 2) % kChunks) * kChunkBytes;
+        if (big) {
+          const int kx = it.kb * BK;
+          tma_load_2d_pair_hint(c0, &p.a_maps[it.am], full_addr, kx, it.a_row, pol_a);
+          tma_load_2d_pair_hint(c1, &p.a_maps[it.am], full_addr, kx, it.a_row + BM, pol_a);
+          tma_load_2d_pair_hint(c2, &p.b_maps[it.bm], full_addr, kx, it.b_row, pol_b);
+        } else {
+          const int kx = it.kb * 2 * BK;
+          uint8_t* c3 = smem + ((chunk + 3) % kChunks) * kChunkBytes;
+          tma_load_2d_pair_hint(c0, &p.a_maps[it.am], full_addr, kx, it.a_row, pol_a);
+          tma_load_2d_pair_hint(c2, &p.b_maps[it.bm], full_addr, kx, it.b_row, pol_b);
+          tma_load_2d_pair_hint(c1, &p.a_maps[it.am], full_addr, kx + BK, it.a_row, pol_a);
+          tma_load_2d_pair_hint(c3, &p.b_maps[it.bm], full_addr, kx + BK, it.b_row, pol_b);
+        }
+        chunk = (chunk + nchunks) % kChunks;
+      }
+      // wait until the last stages have been consumed (the leader's MMAs read both CTAs' chunks)
+      const uint32_t back = j < 4u ? j : 4u;
+      for (uint32_t i = 1; i <= back; ++i) {
+        const uint32_t r = j - i;
+        if (!wait_bounded_m(&ctl->empty[r & 3u], (r >> 2) & 1u, ctl, p, WAIT_DRAIN, -1)) break;
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    // One lane runs the whole loop: a per-instruction "if (lane == 0)" inside a
+    // 32-lane loop costs a divergence per MMA and measurably slows the issue stream.
+    if (leader && lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(2 * BM, BN);
+      const uint64_t desc0 = umma_smem_desc_sw128(smem_u32(smem));
+      uint32_t j = 0;
+      int chunk = 0;
+      uint32_t uses0 = 0, uses1 = 0;      // completed uses of accumulator 0 / 1
+      uint32_t small_rr = 0;
+      bool ok = true;
+      for (int t = unit; ok && t < p.total_tiles; t += n_units) {
+        const MixedTile tile = decode_mixed(p, t);
+        if (!tile.valid) continue;
+        const int big = tile.big;
+        const int kb_seg = big ? p.kb_big : p.kb_per_seg;
+        const int n_kb = kb_seg * p.n_seg;
+        const int tail = big ? p.tail_big : p.tail_ksteps;
+        const uint32_t buf = big ? 0u : (small_rr & 1u);
+        // the accumulator(s) this tile writes must have been drained by the epilogue
+        if (!wait_bounded_m(&ctl->acc_empty[buf], ((buf ? uses1 : uses0) & 1u) ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
+        if (big && !wait_bounded_m(&ctl->acc_empty[1], (uses1 & 1u) ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
+        tc_fence_after_sync();
+        const uint32_t acc_a = tmem_base + buf * BN;
+        int kb_in_seg = 0;
+        for (int kb = 0; kb < n_kb; ++kb, ++j) {
+          if (!wait_bounded_m(&ctl->full[j & 3u], (j >> 2) & 1u, ctl, p, WAIT_SMEM_FULL, t)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after_sync();
+          const bool full_stage = kb_in_seg != kb_seg - 1 || tail == 2 * BK / UMMA_K || (big && tail == BK / UMMA_K);
+          const uint64_t d0 = desc0 + uint64_t((((chunk + 0) % kChunks) * kChunkBytes) >> 4);
+          const uint64_t d1 = desc0 + uint64_t((((chunk + 1) % kChunks) * kChunkBytes) >> 4);
+          const uint64_t d2 = desc0 + uint64_t((((chunk + 2) % kChunks) * kChunkBytes) >> 4);
+          const uint32_t first = kb != 0 ? 1u : 0u;
+          if (big) {
+            // A block 0 -> accumulator 0, A block 1 -> accumulator 1.  The two MMAs of a
+            // k-step are adjacent so that they read the same B slice back to back.
+            if (full_stage) {
+#pragma unroll
+              for (int k = 0; k < BK / UMMA_K; ++k) {
+                umma_bf16_pair(tmem_base, d0 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
+                umma_bf16_pair(tmem_base + BN, d1 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
+              }
+            } else {
+              for (int k = 0; k < tail; ++k) {
+                umma_bf16_pair(tmem_base, d0 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
+                umma_bf16_pair(tmem_base + BN, d1 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
+              }
+            }
+            chunk = (chunk + 3) % kChunks;
+          } else {
+            const uint64_t d3 = desc0 + uint64_t((((chunk + 3) % kChunks) * kChunkBytes) >> 4);
+            if (full_stage) {
+#pragma unroll
+              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc_a, d0 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
+#pragma unroll
+              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc_a, d1 + uint64_t(k * 2), d3 + uint64_t(k * 2), idesc, 1u);
+            } else {
+              for (int ks = 0; ks < tail; ++ks) {
+                const int k = ks & 3;
+                umma_bf16_pair(acc_a, ((ks >> 2) ? d1 : d0) + uint64_t(k * 2), ((ks >> 2) ? d3 : d2) + uint64_t(k * 2), idesc,
+                               ks ? 1u : first);
+              }
+            }
+            chunk = (chunk + 4) % kChunks;
+          }
+          umma_commit_pair(&ctl->empty[j & 3u], 0x3);      // the stage is reusable in both CTAs once these MMAs have read it
+          if (++kb_in_seg == kb_seg) kb_in_seg = 0;
+        }
+        if (!ok) break;
+        if (big) {
+          umma_commit_pair(&ctl->acc_full[0], 0x3);
+          umma_commit_pair(&ctl->acc_full[1], 0x3);
+          ++uses0;
+          ++uses1;
+        } else {
+          umma_commit_pair(&ctl->acc_full[buf], 0x3);
+          if (buf) ++uses1; else ++uses0;
+          ++small_rr;
+        }
+      }
+      if (*reinterpret_cast<volatile int*>(&ctl->abort)) {
+        // gave up somewhere: let the tensor core finish what it still has before tensor memory is released
+        umma_commit_pair(&ctl->drain, 0x1);
+        wait_bounded_m(&ctl->drain, 0, ctl, p, WAIT_DRAIN, -2);
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int quarter = warp & 3;
+    uint8_t* stage = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ctl + 1) + 15) & ~uintptr_t(15)) +
+                     (warp - 2) * kStageWarpBytes;
+    uint32_t uses0 = 0, uses1 = 0, small_rr = 0;
+    bool ok = true;
+    for (int t = unit; ok && t < p.total_tiles; t += n_units) {
+      const MixedTile tile = decode_mixed(p, t);
+      if (!tile.valid) continue;
+      const BlockDesc& b = p.blocks[tile.blk];
+      const int ncols = min(BN, p.N - tile.nt * BN);
+      const int nchunks = (ncols + 31) >> 5;
+      const int n_acc = tile.big ? 2 : 1;
+      for (int a = 0; a < n_acc && ok; ++a) {
+        const uint32_t buf = tile.big ? uint32_t(a) : (small_rr & 1u);
+        const uint32_t n = buf ? uses1 : uses0;
+        if (!wait_bounded_m(&ctl->acc_full[buf], n & 1u, ctl, p, WAIT_ACC_FULL, t)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after_sync();
+        // big: this CTA owns rows [256*rank, +256) of the tile, accumulator a holds its 128-row block a
+        const int row_in_block = tile.row0 + (tile.big ? int(cta_rank) * 2 * BM + a * BM : int(cta_rank) * BM) + quarter * 32 + lane;
+        const bool row_ok = row_in_block < p.rows_per_block;
+        __nv_bfloat16* orow = p.out[b.out_idx] + int64_t(b.out_row0 + row_in_block) * p.ldo + int64_t(tile.nt) * BN;
+        const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
+        const int first_row = row_in_block - lane;          // row of lane 0
+        __nv_bfloat16* obase = orow - int64_t(lane) * p.ldo;
+        const int npass = (ncols + 63) >> 6;
+        for (int pass = 0; pass < npass; ++pass) {
+          // 32 lanes (rows) x 64 columns: TMEM -> registers -> BF16 -> padded shared memory ...
+          uint32_t v[32], w[32];
+          tmem_ld_32x32b_x32(taddr + pass * 64, v);
+          tmem_ld_32x32b_x32(taddr + pass * 64 + 32, w);
+          tmem_ld_wait();
+          if (pass == npass - 1) {
+            // accumulator fully copied out: hand it back to the MMA issuer
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->acc_empty[buf]), 0));
+          }
+          uint4* srow = reinterpret_cast<uint4*>(stage + lane * kStageRowBytes);
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            uint4 q;
+            q.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
+            q.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
+            q.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
+            q.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
+            srow[g] = q;
+            uint4 r;
+            r.x = pack_bf16x2(__uint_as_float(w[g * 8 + 0]), __uint_as_float(w[g * 8 + 1]));
+            r.y = pack_bf16x2(__uint_as_float(w[g * 8 + 2]), __uint_as_float(w[g * 8 + 3]));
+            r.z = pack_bf16x2(__uint_as_float(w[g * 8 + 4]), __uint_as_float(w[g * 8 + 5]));
+            r.w = pack_bf16x2(__uint_as_float(w[g * 8 + 6]), __uint_as_float(w[g * 8 + 7]));
+            srow[4 + g] = r;
+          }
+          __syncwarp();
+          // ... -> global: every instruction writes 4 rows x 128 contiguous bytes
+          const int seg = lane & 7;
+          const int col = pass * 64 + seg * 8;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int r = i * 4 + (lane >> 3);
+            if (first_row + r < p.rows_per_block && col < ncols) {
+              const uint4 q = *reinterpret_cast<const uint4*>(stage + r * kStageRowBytes + seg * 16);
+              *reinterpret_cast<uint4*>(obase + int64_t(r) * p.ldo + col) = q;
+            }
+          }
+          __syncwarp();
+        }
+        if (buf) ++uses1; else ++uses0;
+      }
+      if (!tile.big) ++small_rr;
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
 // ---- host side ----------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -519,6 +897,8 @@ int device_info(DeviceInfo** out) {
     if (e != cudaSuccess) return record_cuda_error(e);
     e = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<true>()));
     if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaFuncSetAttribute(gemm_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kMixedSmemBytes));
+    if (e != cudaSuccess) return record_cuda_error(e);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(unsigned(info.num_sms / 2 * 2));
     cfg.blockDim = dim3(kThreads);
@@ -542,7 +922,10 @@ int device_info(DeviceInfo** out) {
 
 }  // namespace
 
-size_t gemm_smem_bytes() { return smem_bytes<true>() > smem_bytes<false>() ? smem_bytes<true>() : smem_bytes<false>(); }
+size_t gemm_smem_bytes() {
+  size_t m = smem_bytes<true>() > smem_bytes<false>() ? smem_bytes<true>() : smem_bytes<false>();
+  return m > kMixedSmemBytes ? m : kMixedSmemBytes;
+}
 
 int gemm_tile_rows(int mode, int rows_per_block) {
   const bool pair = mode == GEMM_MODE_PAIR || (mode == GEMM_MODE_AUTO && rows_per_block >= 2 * BM);
@@ -589,13 +972,24 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   int st = device_info(&info);
   if (st != COMPASS_OK) return st;
   if (p.total_tiles <= 0) return COMPASS_OK;
+  // Mixed tiles: 512x256 for as many whole waves of pairs as the launch holds, 256x256 for the rest.
+  const bool mixed = pair && info->max_pairs > 0 && L.epilogue == EPI_STORE && L.mode != GEMM_MODE_PAIR;
+  if (mixed) {
+    p.big_tiles_m = (L.rows_per_block + 4 * BM - 1) / (4 * BM);
+    const int total_big = L.n_blocks * p.big_tiles_m * p.tiles_n;
+    const bool use_big = L.rows_per_block % (4 * BM) == 0;
+    p.n_big = use_big ? (total_big / info->max_pairs) * info->max_pairs : 0;
+    p.total_tiles = p.n_big + 2 * (total_big - p.n_big);
+    p.kb_big = int32_t((L.K + BK - 1) / BK);
+    p.tail_big = int32_t((L.K - int64_t(p.kb_big - 1) * BK + UMMA_K - 1) / UMMA_K);
+  }
   cudaError_t e;
   if (pair && info->max_pairs > 0) {
     const int pairs = p.total_tiles < info->max_pairs ? p.total_tiles : info->max_pairs;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(unsigned(2 * pairs));
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem_bytes<true>();
+    cfg.dynamicSmemBytes = mixed ? kMixedSmemBytes : smem_bytes<true>();
     cfg.stream = stream;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
@@ -604,7 +998,7 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, gemm_kernel<true>, p);
+    e = mixed ? cudaLaunchKernelEx(&cfg, gemm_mixed_kernel, p) : cudaLaunchKernelEx(&cfg, gemm_kernel<true>, p);
   } else {
     if (pair) {   // no room for clusters on this device: fall back to single-CTA tiles
       p.tiles_m = (L.rows_per_block + BM - 1) / BM;

@@ -56,6 +56,7 @@ enum GemmMode : int32_t {
   GEMM_MODE_AUTO = 0,     // CTA pairs when a block has at least 256 rows
   GEMM_MODE_SINGLE = 1,   // one CTA per 128x256 tile
   GEMM_MODE_PAIR = 2,     // two CTAs per 256x256 tile
+  GEMM_MODE_MIXED = 3,    // CTA pairs: 512x256 tiles for the full waves, 256x256 for the tail
 };
 
 enum EpilogueMode : int32_t {
@@ -76,6 +77,11 @@ struct GemmParams {
   int32_t tail_ksteps;     // UMMA_K steps in the last k-stage of a segment
   int32_t tiles_m, tiles_n;
   int32_t total_tiles;
+  // mixed-tile pair kernel: tiles [0, n_big) are 512x256, the rest 256x256 (two per remaining big tile)
+  int32_t n_big;
+  int32_t big_tiles_m;     // 512-row tiles per block
+  int32_t kb_big;          // 64-wide k-stages per segment of a big tile
+  int32_t tail_big;        // UMMA_K steps in its last stage
   int32_t epilogue;        // EpilogueMode
   int32_t last_step;       // ring RMW: step index of the final contributor (P-1)
   uint32_t wait_limit_us;  // bound of every device-side wait
