@@ -785,48 +785,49 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
         const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
         const int first_row = row_in_block - lane;          // row of lane 0
         __nv_bfloat16* obase = orow - int64_t(lane) * p.ldo;
-        const int npass = (ncols + 63) >> 6;
-        for (int pass = 0; pass < npass; ++pass) {
-          // 32 lanes (rows) x 64 columns: TMEM -> registers -> BF16 -> padded shared memory ...
+        // 1) The whole accumulator row (256 columns) goes TMEM -> registers as packed BF16, then the
+        //    accumulator is handed back at once: with two live accumulators per tile the MMA issuer
+        //    waits for this, so the time TMEM is held matters more than the time the stores take.
+        uint32_t packed[BN / 2];
+#pragma unroll
+        for (int c = 0; c < BN / 64; ++c) {
           uint32_t v[32], w[32];
-          tmem_ld_32x32b_x32(taddr + pass * 64, v);
-          tmem_ld_32x32b_x32(taddr + pass * 64 + 32, w);
+          tmem_ld_32x32b_x32(taddr + c * 64, v);
+          tmem_ld_32x32b_x32(taddr + c * 64 + 32, w);
           tmem_ld_wait();
-          if (pass == npass - 1) {
-            // accumulator fully copied out: hand it back to the MMA issuer
-            tc_fence_before_sync();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            packed[c * 32 + i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+            packed[c * 32 + 16 + i] = pack_bf16x2(__uint_as_float(w[2 * i]), __uint_as_float(w[2 * i + 1]));
+          }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->acc_empty[buf]), 0));
+        // 2) registers -> padded shared memory -> global, 64 columns per pass: every store
+        //    instruction writes 4 rows x 128 contiguous bytes.
+        const int npass = (ncols + 63) >> 6;
+        const int seg = lane & 7;
+#pragma unroll
+        for (int pass = 0; pass < BN / 64; ++pass) {
+          if (pass < npass) {
+            uint4* srow = reinterpret_cast<uint4*>(stage + lane * kStageRowBytes);
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+              srow[g] = make_uint4(packed[pass * 32 + g * 4 + 0], packed[pass * 32 + g * 4 + 1], packed[pass * 32 + g * 4 + 2],
+                                   packed[pass * 32 + g * 4 + 3]);
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->acc_empty[buf]), 0));
-          }
-          uint4* srow = reinterpret_cast<uint4*>(stage + lane * kStageRowBytes);
+            const int col = pass * 64 + seg * 8;
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint4 q;
-            q.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
-            q.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
-            q.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
-            q.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
-            srow[g] = q;
-            uint4 r;
-            r.x = pack_bf16x2(__uint_as_float(w[g * 8 + 0]), __uint_as_float(w[g * 8 + 1]));
-            r.y = pack_bf16x2(__uint_as_float(w[g * 8 + 2]), __uint_as_float(w[g * 8 + 3]));
-            r.z = pack_bf16x2(__uint_as_float(w[g * 8 + 4]), __uint_as_float(w[g * 8 + 5]));
-            r.w = pack_bf16x2(__uint_as_float(w[g * 8 + 6]), __uint_as_float(w[g * 8 + 7]));
-            srow[4 + g] = r;
-          }
-          __syncwarp();
-          // ... -> global: every instruction writes 4 rows x 128 contiguous bytes
-          const int seg = lane & 7;
-          const int col = pass * 64 + seg * 8;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int r = i * 4 + (lane >> 3);
-            if (first_row + r < p.rows_per_block && col < ncols) {
-              const uint4 q = *reinterpret_cast<const uint4*>(stage + r * kStageRowBytes + seg * 16);
-              *reinterpret_cast<uint4*>(obase + int64_t(r) * p.ldo + col) = q;
+            for (int i = 0; i < 8; ++i) {
+              const int r = i * 4 + (lane >> 3);
+              if (first_row + r < p.rows_per_block && col < ncols) {
+                const uint4 q = *reinterpret_cast<const uint4*>(stage + r * kStageRowBytes + seg * 16);
+                *reinterpret_cast<uint4*>(obase + int64_t(r) * p.ldo + col) = q;
+              }
             }
+            __syncwarp();
           }
-          __syncwarp();
         }
         if (buf) ++uses1; else ++uses0;
       }
