@@ -37,8 +37,8 @@ NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # DRAM bytes (read + written) per launch of the GEMM kernel from the ncu capture summarised in
-# profiles/gemm_kernel_pair_k128_C2_C3.md.
-NCU_TRAFFIC_BYTES = {"C2": 316.6e6, "C3": 1024.0e6}
+# profiles/gemm_mixed_kernel_C2_C3.md.
+NCU_TRAFFIC_BYTES = {"C2": 359.1e6, "C3": 830.9e6}
 
 
 def env_int(name, default):
@@ -479,7 +479,7 @@ def run_ours(args, w_ag, w_rs):
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                          "frac": achieved / peak, "traffic": traffic,
                          "peak_source": f"{'sustained' if sustained else 'burst'} cuBLAS bf16, of {peak_src}",
-                         "kernel": "gemm_kernel (two launches per step: AG-GEMM and GEMM-RS)",
+                         "kernel": "gemm_mixed_kernel (two launches per step: AG-GEMM and GEMM-RS)",
                          "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS},
             "ag_gemm": {"ms": t_ag, "tflops": w_ag.flops / (t_ag * 1e-3) / 1e12,
                         "frac_of_nominal_2250": w_ag.flops / (t_ag * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS},
