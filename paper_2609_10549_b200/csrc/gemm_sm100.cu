@@ -1,4 +1,4 @@
-// Table-driven persistent BF16 GEMM for sm_100a (tcgen05 + TMEM + TMA).
+// Table-driven persistent BF16 GEMMs for sm_100a (tcgen05 + TMEM + TMA).
 //
 // One launch executes a list of "blocks" (contiguous output row ranges, for the
 // fused operators one block = one entry of the ring chunk schedule, Section
@@ -13,21 +13,23 @@
 //   GEMM+ReduceScatter, ring read-modify-write: every rank's partial tile is
 //     added by the epilogue into the owner's rows in ring order.
 //
-// Two modes of the same kernel:
-//   pair   (default when a block has >= 256 rows): a cluster of two CTAs owns a
-//          256x256 tile.  Each CTA loads its 128 rows of A and its 128 rows of B
-//          (64 KB per 128-wide k-stage, 3 stages); the leader CTA issues
-//          tcgen05.mma.cta_group::2, which reads both CTAs' shared memory, and
-//          each CTA's tensor memory receives its 128 rows of the accumulator.
-//          Operand traffic L2 -> SM per flop is 2/3 of the single-CTA form.
-//   single one CTA owns a 128x256 tile (48 KB per k-block, 4 stages); used for
-//          row fragments.
+// Three kernels share the roles and the barrier protocol:
+//   gemm_mixed_kernel  clusters of two CTAs; 512x256 tiles (two accumulators per
+//                      CTA sharing one B tile) for the whole waves of a launch,
+//                      256x256 tiles for the tail; plain-store epilogue.  The
+//                      default for blocks of >= 256 rows.
+//   gemm_kernel<true>  clusters of two CTAs, 256x256 tiles; carries the ring
+//                      read-modify-write epilogue.
+//   gemm_kernel<false> one CTA per 128x256 tile; row fragments below 256 rows.
+// In the pair kernels each CTA loads its own rows of A and its half of the B
+// rows; the leader CTA issues tcgen05.mma.cta_group::2, which reads both CTAs'
+// shared memory, and each CTA's tensor memory receives its rows of the
+// accumulator.  No TMA load uses cluster multicast.
 //
 // Warp roles (192 threads, 1 CTA per SM): warp 0 = TMA producer (one lane),
 // warp 1 = tensor-memory allocation + MMA issue (one lane), warps 2..5 =
-// epilogue (warp w reads TMEM lanes 32*(w%4)..+31).  Two 256-column TMEM
-// accumulators let the epilogue of tile i overlap the main loop of tile i+1.
-// Every wait is bounded and reports COMPASS_ERR_TIMEOUT instead of hanging.
+// epilogue (warp w reads TMEM lanes 32*(w%4)..+31).  Every wait is bounded and
+// reports COMPASS_ERR_TIMEOUT instead of hanging.
 #include "internal.h"
 #include "ptx_sm100.cuh"
 
@@ -40,7 +42,7 @@ namespace {
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;           // two BN-column FP32 accumulators
 constexpr int kEpilogueWarps = 4;
-constexpr int kMaxStages = 7;
+constexpr int kSlots = 4;                      // pipeline barrier pairs (>= stages of every kernel below)
 
 template <bool kPair>
 struct Cfg {
@@ -63,8 +65,8 @@ struct Cfg {
 };
 
 struct Control {
-  uint64_t full[kMaxStages];
-  uint64_t empty[kMaxStages];
+  uint64_t full[kSlots];
+  uint64_t empty[kSlots];
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
   uint64_t drain;
@@ -474,22 +476,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 // 3 for small stages), which also holds across the change of kind.
 constexpr int kChunkBytes = BM * BK * 2;      // 16 KB: one 128-row, 64-column BF16 box
 constexpr int kChunks = 12;
-constexpr int kSlots = 4;
-
-struct MixedControl {
-  uint64_t full[kSlots];
-  uint64_t empty[kSlots];
-  uint64_t acc_full[2];
-  uint64_t acc_empty[2];
-  uint64_t drain;
-  uint32_t tmem_base;
-  int abort;
-};
 // epilogue staging: per epilogue warp 32 rows x 64 BF16 columns, rows padded by 16 bytes (conflict-free 16-byte accesses)
 constexpr int kStageRowBytes = 64 * 2 + 16;
 constexpr int kStageWarpBytes = 32 * kStageRowBytes;
 constexpr size_t kMixedSmemBytes =
-    1024 + size_t(kChunks) * kChunkBytes + sizeof(MixedControl) + 16 + size_t(kEpilogueWarps) * kStageWarpBytes;
+    1024 + size_t(kChunks) * kChunkBytes + sizeof(Control) + 16 + size_t(kEpilogueWarps) * kStageWarpBytes;
 
 struct MixedTile {
   int big;        // 1 = 512x256, 0 = 256x256
@@ -561,36 +552,11 @@ struct MixedIter {
   }
 };
 
-__device__ __forceinline__ void report_timeout_m(const GemmParams& p, MixedControl* ctl, int site, int tile) {
-  *reinterpret_cast<volatile int*>(&ctl->abort) = 1;
-  if (atomicCAS(&p.status->code, 0, int(COMPASS_ERR_TIMEOUT)) == 0) {
-    p.status->detail = site;
-    p.status->block_idx = int(blockIdx.x);
-    p.status->tile = tile;
-  }
-}
-__device__ __forceinline__ bool wait_bounded_m(uint64_t* bar, uint32_t parity, MixedControl* ctl, const GemmParams& p, int site,
-                                               int tile) {
-  if (mbar_test_wait(bar, parity)) return true;
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = globaltimer_ns();
-  const uint64_t limit = uint64_t(p.wait_limit_us) * 1000ull;
-  for (uint32_t spins = 1; spins < (1u << 30); ++spins) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((spins & 0xFF) == 0) {
-      if (*reinterpret_cast<volatile int*>(&ctl->abort)) return false;
-      if (globaltimer_ns() - t0 > limit) break;
-    }
-  }
-  report_timeout_m(p, ctl, site, tile);
-  return false;
-}
-
 __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   uint8_t* smem = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
-  MixedControl* ctl = reinterpret_cast<MixedControl*>(smem + kChunks * kChunkBytes);
+  Control* ctl = reinterpret_cast<Control*>(smem + kChunks * kChunkBytes);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -635,7 +601,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
         const uint32_t depth = big ? 4u : 3u;
         if (j >= depth) {
           const uint32_t r = j - depth;      // this stage's chunks are free once stage r has been released
-          if (!wait_bounded_m(&ctl->empty[r & 3u], (r >> 2) & 1u, ctl, p, WAIT_SMEM_EMPTY, it.t)) break;
+          if (!wait_bounded(&ctl->empty[r & 3u], (r >> 2) & 1u, ctl, p, WAIT_SMEM_EMPTY, it.t)) break;
         }
         const uint32_t slot = j & 3u;
         const uint32_t full_addr = map_to_cta(smem_u32(&ctl->full[slot]), 0);
@@ -663,7 +629,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
       const uint32_t back = j < 4u ? j : 4u;
       for (uint32_t i = 1; i <= back; ++i) {
         const uint32_t r = j - i;
-        if (!wait_bounded_m(&ctl->empty[r & 3u], (r >> 2) & 1u, ctl, p, WAIT_DRAIN, -1)) break;
+        if (!wait_bounded(&ctl->empty[r & 3u], (r >> 2) & 1u, ctl, p, WAIT_DRAIN, -1)) break;
       }
     }
   } else if (warp == 1) {
@@ -687,13 +653,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
         const int tail = big ? p.tail_big : p.tail_ksteps;
         const uint32_t buf = big ? 0u : (small_rr & 1u);
         // the accumulator(s) this tile writes must have been drained by the epilogue
-        if (!wait_bounded_m(&ctl->acc_empty[buf], ((buf ? uses1 : uses0) & 1u) ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
-        if (big && !wait_bounded_m(&ctl->acc_empty[1], (uses1 & 1u) ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
+        if (!wait_bounded(&ctl->acc_empty[buf], ((buf ? uses1 : uses0) & 1u) ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
+        if (big && !wait_bounded(&ctl->acc_empty[1], (uses1 & 1u) ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
         tc_fence_after_sync();
         const uint32_t acc_a = tmem_base + buf * BN;
         int kb_in_seg = 0;
         for (int kb = 0; kb < n_kb; ++kb, ++j) {
-          if (!wait_bounded_m(&ctl->full[j & 3u], (j >> 2) & 1u, ctl, p, WAIT_SMEM_FULL, t)) {
+          if (!wait_bounded(&ctl->full[j & 3u], (j >> 2) & 1u, ctl, p, WAIT_SMEM_FULL, t)) {
             ok = false;
             break;
           }
@@ -753,7 +719,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
       if (*reinterpret_cast<volatile int*>(&ctl->abort)) {
         // gave up somewhere: let the tensor core finish what it still has before tensor memory is released
         umma_commit_pair(&ctl->drain, 0x1);
-        wait_bounded_m(&ctl->drain, 0, ctl, p, WAIT_DRAIN, -2);
+        wait_bounded(&ctl->drain, 0, ctl, p, WAIT_DRAIN, -2);
       }
     }
   } else {
@@ -773,7 +739,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
       for (int a = 0; a < n_acc && ok; ++a) {
         const uint32_t buf = tile.big ? uint32_t(a) : (small_rr & 1u);
         const uint32_t n = buf ? uses1 : uses0;
-        if (!wait_bounded_m(&ctl->acc_full[buf], n & 1u, ctl, p, WAIT_ACC_FULL, t)) {
+        if (!wait_bounded(&ctl->acc_full[buf], n & 1u, ctl, p, WAIT_ACC_FULL, t)) {
           ok = false;
           break;
         }

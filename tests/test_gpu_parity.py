@@ -84,6 +84,29 @@ def test_gemm_rs_small_shapes(P, m, N, K, rings):
     check_all(outs, ops.gemm_rs(A, B, rings=rings), w.name)
 
 
+# Enough 512-row partitions to fill whole waves of CTA pairs with 512x256 tiles and leave a
+# tail of 256x256 tiles, with ragged N (2568 = 10 tiles + 8 columns) and a K tail; checked
+# element by element.
+@pytest.mark.parametrize("op,P,m,N,K,order", [
+    (wl.OP_AG_GEMM, 4, 1024, 2568, 200, api.ORDER_RANK_MAJOR),
+    (wl.OP_AG_GEMM, 4, 1024, 2568, 72, api.ORDER_STEP_MAJOR),
+    (wl.OP_GEMM_RS, 8, 1024, 2568, 88, api.ORDER_RANK_MAJOR),
+    (wl.OP_AG_GEMM, 2, 1536, 5128, 64, api.ORDER_RANK_MAJOR),      # 768-row partitions: 512-row tiles do not divide them
+])
+def test_big_and_small_tiles_in_one_launch(op, P, m, N, K, order):
+    w = small(op, P, m, N, K, dist=0.05)
+    A_bits, B_bits = wl.make_inputs(w)
+    pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, order=order)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    ws = api.alloc_workspace(pr)
+    (api.compass_ag_gemm if op == wl.OP_AG_GEMM else api.compass_gemm_rs)(pr, A, B, [o.view for o in outs], ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    assert all(o.guards_intact() for o in outs)
+    refs = ops.ag_gemm(A_bits, B_bits) if op == wl.OP_AG_GEMM else ops.gemm_rs(A_bits, B_bits)
+    check_all([o.bits() for o in outs], refs, w.name)
+
+
 @pytest.mark.parametrize("op", [wl.OP_AG_GEMM, wl.OP_GEMM_RS])
 def test_integer_inputs_are_reproduced_exactly(op):
     """Small-integer inputs make every partial sum exact in FP32 and every
