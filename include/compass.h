@@ -82,7 +82,9 @@ enum { COMPASS_STRATEGY_INTRAFUSION = 0, COMPASS_STRATEGY_INTERDECOM = 1 };
  *     shard stays in L2 while it is used; default);
  *   STEP_MAJOR: all ranks advance in lockstep: step 0 of every rank, then
  *     step 1, ... (what P GPUs running concurrently would do).
- * The ring read-modify-write variant always uses STEP_MAJOR. */
+ * The ring read-modify-write variant always uses STEP_MAJOR (its ordered adds
+ * need contributor s of a partition to precede contributor s+1 in the launch);
+ * the segmented-K variant has one block per partition and ignores the field. */
 enum { COMPASS_ORDER_RANK_MAJOR = 0, COMPASS_ORDER_STEP_MAJOR = 1 };
 /* selectors for compass_workspace_bytes */
 enum { COMPASS_WS_FUSED = 0, COMPASS_WS_DECOMP = 1 };
