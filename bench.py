@@ -248,9 +248,17 @@ def interdecom_report(torch, api):
             self.ws = api.alloc_workspace(self.pr)
             self.fused = api.compass_ag_gemm if w.op == wl.OP_AG_GEMM else api.compass_gemm_rs
             self.dws = None
+            self.pws = None
 
         def t_fused(self):
             return median_ms(lambda: self.fused(self.pr, self.A, self.B, self.out, self.ws, stream))
+
+        def t_push(self):
+            """AllGather+GEMM with pushed partitions and readiness flags (the paper's mechanism)."""
+            if self.pws is None:
+                self.pws = torch.empty(api.compass_workspace_bytes(self.pr, api.WS_PUSH), dtype=torch.uint8, device="cuda")
+                api.compass_workspace_init(self.pws)
+            return median_ms(lambda: api.compass_ag_gemm_push(self.pr, self.A, self.B, self.out, self.pws, stream, side))
 
         def t_decomp(self, d):
             pr = api.make_problem(self.w.op, self.w.P, self.w.M, self.w.N, self.w.K, d=d)
@@ -279,14 +287,16 @@ def interdecom_report(torch, api):
             for d in degrees[1:]:
                 if w.m % d == 0:
                     dc.append(t_comp); dm.append(t_comm); dd.append(d); dt.append(c.t_decomp(d))
-            fc.append(t_comp); fm.append(t_comm); fn_.append(w.P); fv.append(c.volume()); ft.append(t_comp)
+            # T_fusion is measured on the variant that really moves the partitions (AG); GEMM+RS has none: its fused
+            # kernel moves no data, so its measured time is T_comp and the fitted overhead comes out ~0.
+            fc.append(t_comp); fm.append(t_comm); fn_.append(w.P); fv.append(c.volume())
+            ft.append(c.t_push() if w.op == wl.OP_AG_GEMM else t_comp)
             del c
             torch.cuda.empty_cache()
         ca, cb = api.compass_calib_fit_line(comp_x, comp_y)
         ma, mb = api.compass_calib_fit_line(comm_x, comm_y)
         alpha, beta = api.compass_calib_fit_decomp(dc, dm, dd, dt)
-        # On one GPU the fused kernel has no transfer to wait for: its measured time *is* T_comp, so the
-        # synchronisation overhead of Eq. 8 is what remains of Eq. 7 after the overlapped terms.
+        # Eq. 8: what remains of the measured fused time after Eq. 7's overlapped terms, per synchronisation point.
         af, bf = api.compass_calib_fit_fusion(fc, fm, fn_, fv, ft)
         return api.Calib(ca, cb, ma, mb, alpha, beta, af, bf)
 
@@ -294,13 +304,18 @@ def interdecom_report(torch, api):
         c = Case(w)
         choice = api.compass_select(c.pr, calib)
         t_fused = c.t_fused()
+        t_push = c.t_push() if w.op == wl.OP_AG_GEMM else None
         ds = [d for d in degrees if w.m % d == 0] if measure_all else sorted({1, choice.d_star})
         times = {d: c.t_decomp(d) for d in ds}
         best_d = min(times, key=times.get)
-        out = {"workload": w.name, "fused_ms": t_fused, "decomp_ms": {str(d): t for d, t in times.items()},
+        # IntraFusion as the paper builds it moves the partitions while it computes: compare that variant with
+        # InterDecom where it exists; the gather-by-address kernel (no transfers at all) is reported beside it.
+        t_intra = t_push if t_push is not None else t_fused
+        out = {"workload": w.name, "fused_ms": t_fused, "push_ms": t_push,
+               "decomp_ms": {str(d): t for d, t in times.items()},
                "measured_best_d": best_d, "predicted_d": choice.d_star,
                "predicted_strategy": "IntraFusion" if choice.strategy == api.STRATEGY_INTRAFUSION else "InterDecom",
-               "measured_winner": "IntraFusion" if t_fused < times[best_d] else "InterDecom",
+               "measured_winner": "IntraFusion" if t_intra < times[best_d] else "InterDecom",
                "model_ms": {"t_comp": choice.t_comp, "t_comm": choice.t_comm, "lambda": choice.lam,
                             "t_decomp": choice.t_decomp, "t_fusion": choice.t_fusion}}
         del c

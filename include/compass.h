@@ -87,7 +87,7 @@ enum { COMPASS_STRATEGY_INTRAFUSION = 0, COMPASS_STRATEGY_INTERDECOM = 1 };
  * the segmented-K variant has one block per partition and ignores the field. */
 enum { COMPASS_ORDER_RANK_MAJOR = 0, COMPASS_ORDER_STEP_MAJOR = 1 };
 /* selectors for compass_workspace_bytes */
-enum { COMPASS_WS_FUSED = 0, COMPASS_WS_DECOMP = 1 };
+enum { COMPASS_WS_FUSED = 0, COMPASS_WS_DECOMP = 1, COMPASS_WS_PUSH = 2 };
 
 /* Workload descriptor W = (pattern, M, N, K, world size[, d]) of Table IV and
  * Algorithm 1.  See the header comment for the meaning of M, N, K per op. */
@@ -166,6 +166,26 @@ int compass_schedule(int op, int P, int rings, int64_t M,
 int compass_ag_gemm(const compass_problem* problem, const void* const* A, const void* const* B,
                     void* const* C, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* ---- fused AllGather+GEMM driven by data readiness (Section III-B) --------
+ * The paper's mechanism itself -- push-based transfers by the DMA engines plus
+ * semaphores that the GEMM tiles wait on -- emulated on one GPU.  Every rank r
+ * has a private gather buffer G_r [M x K] in the workspace.  On stream_copy,
+ * step by step (s = 1 .. P-1) and ring by ring, the partition that rank r
+ * processes at step s is pushed by a device-to-device copy from its upstream
+ * neighbour (from the neighbour's shard at s = 1, from the neighbour's gather
+ * buffer afterwards: hop by hop, as on the ring) into G_r, and a readiness
+ * flag is raised in stream order behind the copy.  ONE GEMM kernel on
+ * stream_compute runs concurrently: step-0 tiles read the local shard at once
+ * and hide the first transfers; a tile of a later step is loaded only after
+ * its partition's flag is up (bounded wait; a wait that gives up reports
+ * COMPASS_ERR_TIMEOUT).  Tiles are issued step-major (all ranks in lockstep).
+ * Arguments as compass_ag_gemm; workspace >= compass_workspace_bytes(problem,
+ * COMPASS_WS_PUSH).  On return all work is ordered before later work on
+ * stream_compute.  stream_copy must differ from stream_compute. */
+int compass_ag_gemm_push(const compass_problem* problem, const void* const* A, const void* const* B,
+                         void* const* C, void* workspace, size_t workspace_bytes,
+                         void* stream_compute, void* stream_copy);
+
 /* ---- fused GEMM+ReduceScatter (Section III-B, last paragraph) ------------
  * ONE kernel launch, no separate reduce kernel.  For partition p = (chunk c,
  * ring g) the contributions are added in the order in which the running sum
@@ -223,8 +243,8 @@ int compass_calib_fit_fusion(const double* t_comp, const double* t_comm, const i
                              const double* t_measured, size_t n, double* alpha_f, double* beta_f);
 
 /* ---- helpers ------------------------------------------------------------- */
-/* Workspace size in bytes for the fused call (which = COMPASS_WS_FUSED) or for
- * compass_decomp (COMPASS_WS_DECOMP) of this problem. */
+/* Workspace size in bytes for the fused call (which = COMPASS_WS_FUSED), for
+ * compass_decomp (COMPASS_WS_DECOMP) or for compass_ag_gemm_push (COMPASS_WS_PUSH). */
 int compass_workspace_bytes(const compass_problem* problem, int which, size_t* bytes);
 /* Zero the status block and every counter of a workspace (asynchronous). */
 int compass_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream);

@@ -23,7 +23,7 @@ DTYPE_BF16 = 0
 RS_SEGMENTED_K, RS_RING_RMW = 0, 1
 STRATEGY_INTRAFUSION, STRATEGY_INTERDECOM = 0, 1
 ORDER_RANK_MAJOR, ORDER_STEP_MAJOR = 0, 1
-WS_FUSED, WS_DECOMP = 0, 1
+WS_FUSED, WS_DECOMP, WS_PUSH = 0, 1, 2
 MAX_P = 16
 STATUS_BYTES = 256
 
@@ -34,7 +34,7 @@ EXPORTS = (
     "compass_calib_fit_decomp", "compass_calib_fit_fusion", "compass_workspace_bytes", "compass_workspace_init",
     "compass_read_status", "compass_launch_plan", "compass_fused_host", "compass_status_string",
     "compass_last_cuda_error", "compass_kernel_launch_count", "compass_gemm_rs_sequential_noalloc",
-    "compass_set_wait_limit_us", "compass_calib_fit_line",
+    "compass_set_wait_limit_us", "compass_calib_fit_line", "compass_ag_gemm_push",
 )
 
 
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
         for name in ("compass_ag_gemm", "compass_gemm_rs"):
             getattr(L, name).argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p]
         L.compass_decomp.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.compass_ag_gemm_push.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.compass_select.argtypes = [C.POINTER(Problem), C.POINTER(Calib), C.POINTER(Choice)]
         L.compass_model_decomp_time.argtypes = [C.c_double] * 4 + [C.c_int, C.POINTER(C.c_double)]
         L.compass_model_optimal_degree.argtypes = [C.c_double] * 4 + [C.c_int, C.c_int, C.POINTER(C.c_int),
@@ -259,6 +260,13 @@ def compass_gemm_rs(problem: Problem, A: Sequence, B: Sequence, Out: Sequence, w
     p, n = _ws(workspace)
     _check(lib().compass_gemm_rs(C.byref(problem), _ptr_array(A), _ptr_array(B), _ptr_array(Out), p, n,
                                  _stream_handle(stream)), "compass_gemm_rs")
+
+
+def compass_ag_gemm_push(problem: Problem, A: Sequence, B: Sequence, Cout: Sequence, workspace, stream_compute,
+                         stream_copy) -> None:
+    p, n = _ws(workspace)
+    _check(lib().compass_ag_gemm_push(C.byref(problem), _ptr_array(A), _ptr_array(B), _ptr_array(Cout), p, n,
+                                      _stream_handle(stream_compute), _stream_handle(stream_copy)), "compass_ag_gemm_push")
 
 
 def compass_decomp(problem: Problem, A: Sequence, B: Sequence, out: Sequence, workspace, stream_compute=None,

@@ -65,6 +65,9 @@ size_t rmw_counter_count(const compass_problem* pr) {
   return size_t(pr->rings) * size_t(pr->P) * size_t(tiles_of(h, BM)) * size_t(tiles_of(pr->N, BN));
 }
 
+// Readiness flags of the push variant: one per (rank, partition).
+size_t push_flag_count(const compass_problem* pr) { return size_t(pr->P) * size_t(pr->rings) * size_t(pr->P); }
+
 // ---- fused launches: schedule -> blocks -------------------------------------
 
 // AllGather+GEMM: one block per schedule entry, listed step-major, then ring,
@@ -375,16 +378,20 @@ using namespace compass;
 
 extern "C" int compass_workspace_bytes(const compass_problem* pr, int which, size_t* bytes) {
   if (bytes == nullptr) return COMPASS_ERR_INVALID_ARG;
-  if (which != COMPASS_WS_FUSED && which != COMPASS_WS_DECOMP) return COMPASS_ERR_INVALID_ARG;
+  if (which != COMPASS_WS_FUSED && which != COMPASS_WS_DECOMP && which != COMPASS_WS_PUSH) return COMPASS_ERR_INVALID_ARG;
+  if (which == COMPASS_WS_PUSH && pr != nullptr && pr->op != COMPASS_OP_AG_GEMM) return COMPASS_ERR_INVALID_ARG;
   int st = validate_problem(pr, -1, which == COMPASS_WS_DECOMP);
   if (st != COMPASS_OK) return st;
   size_t total = COMPASS_STATUS_BYTES;
   if (which == COMPASS_WS_FUSED) {
     if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant == COMPASS_RS_RING_RMW)
       total += align_up(rmw_counter_count(pr) * sizeof(int32_t));
-  } else {
+  } else if (which == COMPASS_WS_DECOMP) {
     const size_t inner = pr->op == COMPASS_OP_AG_GEMM ? size_t(pr->K) : size_t(pr->N);
     total += size_t(pr->P) * align_up(size_t(pr->M) * inner * 2);
+  } else {
+    total += align_up(push_flag_count(pr) * sizeof(uint32_t));
+    total += size_t(pr->P) * align_up(size_t(pr->M) * size_t(pr->K) * 2);
   }
   *bytes = total;
   return COMPASS_OK;
@@ -433,6 +440,124 @@ extern "C" int compass_ag_gemm(const compass_problem* pr, const void* const* A, 
 extern "C" int compass_gemm_rs(const compass_problem* pr, const void* const* A, const void* const* B, void* const* Out,
                                void* ws, size_t ws_bytes, void* stream) {
   return fused_call(pr, COMPASS_OP_GEMM_RS, A, B, Out, ws, ws_bytes, stream);
+}
+
+// cuStreamWriteValue32: a stream-ordered 32-bit store executed by the front end (no SM, no copy engine).
+typedef CUresult (*StreamWriteValue32Fn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
+static StreamWriteValue32Fn stream_write_fn() {
+  static StreamWriteValue32Fn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<StreamWriteValue32Fn>(ptr);
+  }
+  return fn;
+}
+
+extern "C" int compass_ag_gemm_push(const compass_problem* pr, const void* const* A, const void* const* B, void* const* C,
+                                    void* ws, size_t ws_bytes, void* stream_compute, void* stream_copy) {
+  int st = validate_problem(pr, COMPASS_OP_AG_GEMM, false);
+  if (st != COMPASS_OK) return st;
+  st = validate_pointers(A, B, C, pr->P);
+  if (st != COMPASS_OK) return st;
+  st = validate_workspace(pr, COMPASS_WS_PUSH, ws, ws_bytes);
+  if (st != COMPASS_OK) return st;
+  if (stream_compute == stream_copy) return COMPASS_ERR_INVALID_ARG;
+  StreamWriteValue32Fn write_value = stream_write_fn();
+  if (write_value == nullptr) return COMPASS_ERR_UNSUPPORTED;
+
+  const int P = pr->P, rings = pr->rings;
+  const int64_t m = pr->M / P, h = m / rings, K = pr->K;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  uint32_t* flags = reinterpret_cast<uint32_t*>(base + COMPASS_STATUS_BYTES);
+  const size_t gather_bytes = align_up(size_t(pr->M) * size_t(K) * 2);
+  uint8_t* G[kMaxP];
+  for (int r = 0; r < P; ++r)
+    G[r] = base + COMPASS_STATUS_BYTES + align_up(push_flag_count(pr) * sizeof(uint32_t)) + size_t(r) * gather_bytes;
+
+  static thread_local compass_sched_entry table[kMaxBlocks];
+  build_schedule(COMPASS_OP_AG_GEMM, P, rings, pr->M, table);
+  // A flag is up once it holds this call's token; tokens grow, so flags never need clearing.
+  static std::atomic<uint32_t> epoch{0};
+  const uint32_t token = epoch.fetch_add(1) + 1;
+
+  static thread_local GemmLaunch L;
+  L.n_a = 2 * P;                       // maps 0..P-1: the shards, P..2P-1: the gather buffers
+  L.n_b = L.n_out = P;
+  L.a_rows = m;
+  L.K = K;
+  L.N = pr->N;
+  L.ldo = pr->N;
+  L.n_seg = 1;
+  L.rows_per_block = int(h);
+  L.epilogue = EPI_STORE;
+  L.status = reinterpret_cast<StatusBlock*>(ws);
+  L.flags = flags;
+  L.flag_token = token;
+  for (int r = 0; r < P; ++r) {
+    L.a_ptr[r] = A[r];
+    L.a_map_rows[r] = m;
+    L.a_ptr[P + r] = G[r];
+    L.a_map_rows[P + r] = pr->M;
+    L.b_ptr[r] = B[r];
+    L.out_ptr[r] = C[r];
+  }
+  int n = 0;
+  for (int step = 0; step < P; ++step)
+    for (int ring = 0; ring < rings; ++ring)
+      for (int rank = 0; rank < P; ++rank) {
+        const compass_sched_entry& e = table[(size_t(rank) * P + step) * rings + ring];
+        BlockDesc& b = L.blocks[n++];
+        b = BlockDesc{};
+        if (step == 0) {                       // local data: available at once
+          b.a_map = uint8_t(rank);
+          b.a_row0 = e.row_begin - e.chunk * int32_t(m);
+        } else {                               // arrives in this rank's gather buffer
+          b.a_map = uint8_t(P + rank);
+          b.a_row0 = e.row_begin;
+          b.flag1 = uint16_t(1 + rank * rings * P + e.part);
+        }
+        b.b_map = uint8_t(rank);
+        b.out_idx = uint8_t(rank);
+        b.out_row0 = e.row_begin;
+        b.step = uint8_t(step);
+        b.part = uint8_t(e.part);
+      }
+  L.n_blocks = n;
+
+  cudaStream_t sc = static_cast<cudaStream_t>(stream_compute), sp = static_cast<cudaStream_t>(stream_copy);
+  std::lock_guard<std::mutex> lock(g_events.mu);
+  st = g_events.ensure(2);
+  if (st != COMPASS_OK) return st;
+  cudaError_t e;
+  // the pushes start after whatever precedes this call on the compute stream (inputs ready, buffers free)
+  if ((e = cudaEventRecord(g_events.ev[0], sc)) != cudaSuccess) return record_cuda_error(e);
+  if ((e = cudaStreamWaitEvent(sp, g_events.ev[0], 0)) != cudaSuccess) return record_cuda_error(e);
+  const size_t part_bytes = size_t(h) * size_t(K) * 2;
+  for (int step = 1; step < P; ++step)
+    for (int ring = 0; ring < rings; ++ring)
+      for (int rank = 0; rank < P; ++rank) {
+        const compass_sched_entry& en = table[(size_t(rank) * P + step) * rings + ring];
+        const int peer = en.peer;              // upstream neighbour that pushes the partition
+        const uint8_t* src = (step == 1)
+                                 ? static_cast<const uint8_t*>(A[peer]) + size_t(en.row_begin - en.chunk * m) * size_t(K) * 2
+                                 : G[peer] + size_t(en.row_begin) * size_t(K) * 2;
+        uint8_t* dst = G[rank] + size_t(en.row_begin) * size_t(K) * 2;
+        if ((e = cudaMemcpyAsync(dst, src, part_bytes, cudaMemcpyDeviceToDevice, sp)) != cudaSuccess)
+          return record_cuda_error(e);
+        uint32_t* flag = flags + size_t(rank) * rings * P + en.part;
+        if (write_value(reinterpret_cast<CUstream>(sp), reinterpret_cast<CUdeviceptr>(flag), token, 0) != CUDA_SUCCESS)
+          return record_cuda_error(cudaErrorUnknown);
+      }
+  if ((e = cudaEventRecord(g_events.ev[1], sp)) != cudaSuccess) return record_cuda_error(e);
+  st = launch_gemm(L, sc);
+  if (st != COMPASS_OK) return st;
+  if ((e = cudaStreamWaitEvent(sc, g_events.ev[1], 0)) != cudaSuccess) return record_cuda_error(e);
+  return COMPASS_OK;
 }
 
 extern "C" int compass_decomp(const compass_problem* pr, const void* const* A, const void* const* B, void* const* out,

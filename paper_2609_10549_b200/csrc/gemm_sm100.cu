@@ -123,6 +123,30 @@ __device__ __forceinline__ bool wait_counter(const int* counter, int target, Con
   return false;
 }
 
+// Bounded wait until a pushed partition has arrived: its flag (written in stream order after
+// the copy that fills the rows) holds the launch's token.  The rows were written by a copy
+// engine and are read next through the async proxy (TMA), hence the proxy fence.
+__device__ __forceinline__ bool wait_ready_flag(const GemmParams& p, const BlockDesc& b, Control* ctl, int tile) {
+  if (p.flags == nullptr || b.flag1 == 0) return true;
+  const uint32_t* flag = p.flags + (b.flag1 - 1);
+  const uint64_t t0 = globaltimer_ns();
+  const uint64_t limit = uint64_t(p.wait_limit_us) * 1000ull;
+  for (uint32_t spins = 0; spins < (1u << 30); ++spins) {
+    uint32_t v;
+    asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v >= p.flag_token) {
+      asm volatile("fence.proxy.async;" ::: "memory");
+      return true;
+    }
+    if ((spins & 0x3F) == 0x3F) {
+      if (*reinterpret_cast<volatile int*>(&ctl->abort)) return false;
+      if (globaltimer_ns() - t0 > limit) break;
+    }
+  }
+  report_timeout(p, ctl, WAIT_READY_FLAG, tile);
+  return false;
+}
+
 struct TileCoord {
   int blk, mt, nt;
 };
@@ -233,7 +257,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       StageIter<kPair> ld(p, unit, n_units, int(cta_rank));
       StageIter<kPair> pf(p, unit, n_units, int(cta_rank));
       for (int i = 0; i < p.prefetch_stages && pf.valid(p); ++i) pf.next(p);
+      int ready_t = -1;
       while (ld.valid(p)) {
+        if (ld.t != ready_t) {      // first stage of a tile: its A rows may still be on their way
+          if (!wait_ready_flag(p, p.blocks[decode_tile(p, ld.t).blk], ctl, ld.t)) break;
+          ready_t = ld.t;
+        }
         if (!wait_bounded(&ctl->empty[stage], phase ^ 1u, ctl, p, WAIT_SMEM_EMPTY, ld.t)) break;
         const int kx = ld.kb * C::kStageK;
         if (kPair) {
@@ -596,7 +625,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
       const uint64_t pol_b = make_l2_policy(p.b_hint);
       uint32_t j = 0;          // global stage counter
       int chunk = 0;           // ring cursor
+      int ready_t = -1;
       for (MixedIter it(p, unit, n_units, int(cta_rank)); it.valid(p); it.next(p), ++j) {
+        if (it.t != ready_t) {      // first stage of a tile: its A rows may still be on their way
+          if (!wait_ready_flag(p, p.blocks[it.tile.blk], ctl, it.t)) break;
+          ready_t = it.t;
+        }
         const int big = it.tile.big;
         const uint32_t depth = big ? 4u : 3u;
         if (j >= depth) {
@@ -905,7 +939,8 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   const bool pair = tile_rows == 2 * BM;
   const int b_box_rows = pair ? BN / 2 : BN;
   for (int i = 0; i < L.n_a; ++i)
-    if (!encode_kmajor(&p.a_maps[i], L.a_ptr[i], L.a_rows, L.K, BM)) return record_cuda_error(cudaErrorUnknown);
+    if (!encode_kmajor(&p.a_maps[i], L.a_ptr[i], L.a_map_rows[i] ? L.a_map_rows[i] : L.a_rows, L.K, BM))
+      return record_cuda_error(cudaErrorUnknown);
   for (int i = 0; i < L.n_b; ++i)
     if (!encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, b_box_rows)) return record_cuda_error(cudaErrorUnknown);
   for (int i = 0; i < L.n_out; ++i) p.out[i] = static_cast<__nv_bfloat16*>(L.out_ptr[i]);
@@ -930,6 +965,8 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
 
   p.status = L.status;
   p.tile_counters = L.tile_counters;
+  p.flags = L.flags;
+  p.flag_token = L.flag_token;
   for (int b = 0; b < L.n_blocks; ++b) p.blocks[b] = L.blocks[b];
   if (L.n_seg > 1)
     for (int b = 0; b < L.n_blocks; ++b)

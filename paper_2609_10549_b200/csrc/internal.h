@@ -37,6 +37,7 @@ enum WaitSite : int32_t {
   WAIT_ACC_FULL = 4,       // epilogue waiting for an accumulator
   WAIT_DRAIN = 5,          // teardown waiting for outstanding work
   WAIT_TILE_COUNTER = 6,   // ring read-modify-write waiting for the previous contributor
+  WAIT_READY_FLAG = 7,     // TMA producer waiting for a pushed partition to arrive
 };
 
 // A block is a contiguous range of output rows handled as tiles_m x tiles_n
@@ -49,7 +50,8 @@ struct BlockDesc {
   uint8_t out_idx;    // index of the output pointer
   uint8_t step;       // schedule step (ring read-modify-write: contributor index)
   uint8_t part;       // schedule partition id
-  uint8_t pad[3];
+  uint8_t pad;
+  uint16_t flag1;     // 1 + index of the readiness flag the block's A rows wait for (0 = always ready)
 };
 
 enum GemmMode : int32_t {
@@ -64,8 +66,10 @@ enum EpilogueMode : int32_t {
   EPI_RING_RMW = 1,   // ordered accumulate into the output in ring order
 };
 
+constexpr int kMaxAMaps = 2 * kMaxP;   // shards plus, for the push variant, the per-rank gather buffers
+
 struct GemmParams {
-  CUtensorMap a_maps[kMaxP];
+  CUtensorMap a_maps[kMaxAMaps];
   CUtensorMap b_maps[kMaxP];
   __nv_bfloat16* out[kMaxP];
   int64_t ldo;             // output row pitch in elements
@@ -89,13 +93,16 @@ struct GemmParams {
   int32_t prefetch_stages; // how many k-stages ahead of the shared-memory loads operands are prefetched into L2 (0 = off)
   StatusBlock* status;
   int32_t* tile_counters;  // ring RMW only
+  const uint32_t* flags;   // readiness flags (push variant), else nullptr
+  uint32_t flag_token;     // a flag is up once it holds a value >= this
   uint8_t seg_rank[kMaxSegBlocks][kMaxP];   // segmented-K: tensor index of segment s of block b
   BlockDesc blocks[kMaxBlocks];
 };
 
 // Host-side description of a GEMM launch before tensor maps are encoded.
 struct GemmLaunch {
-  const void* a_ptr[kMaxP];
+  const void* a_ptr[kMaxAMaps];
+  int64_t a_map_rows[kMaxAMaps] = {};   // rows of A tensor i; 0 = a_rows
   const void* b_ptr[kMaxP];
   void* out_ptr[kMaxP];
   int n_a = 0, n_b = 0, n_out = 0;
@@ -117,6 +124,8 @@ struct GemmLaunch {
   uint8_t seg_rank[kMaxSegBlocks][kMaxP];
   StatusBlock* status = nullptr;
   int32_t* tile_counters = nullptr;
+  const uint32_t* flags = nullptr;
+  uint32_t flag_token = 0;
 };
 
 // gemm_sm100.cu

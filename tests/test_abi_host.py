@@ -179,6 +179,8 @@ def test_workspace_sizes():
     assert _codes(ag, api.WS_DECOMP) == (api.OK, api.STATUS_BYTES + 4 * 4096 * 4096 * 2)
     rs = api.make_problem(OP_GEMM_RS, 4, 4096, 4096, 1024, d=2)
     assert _codes(rs, api.WS_DECOMP) == (api.OK, api.STATUS_BYTES + 4 * 4096 * 4096 * 2)
+    assert _codes(ag, api.WS_PUSH) == (api.OK, api.STATUS_BYTES + 256 + 4 * 4096 * 4096 * 2)     # 32 flags + 4 gather buffers
+    assert _codes(rs, api.WS_PUSH)[0] == api.ERR_INVALID_ARG
     ring = api.make_problem(OP_GEMM_RS, 8, 8192, 4096, 1376, rs_variant=api.RS_RING_RMW)
     code, n = _codes(ring)
     assert code == api.OK and n >= api.STATUS_BYTES + 16 * 4 * 16 * 4

@@ -296,3 +296,58 @@ def test_bounded_wait_reports_timeout_and_the_context_survives():
     api.compass_gemm_rs(pr, A, B, [o.view for o in outs], ws)
     assert api.compass_read_status(ws) == (api.OK, 0)
     check_ring([o.bits() for o in outs], ops.gemm_rs(A_bits, B_bits), w.name, w.P)
+
+
+# ---- AllGather+GEMM driven by pushed partitions and readiness flags ----------------------------
+
+def run_push(w, A_bits, B_bits, rings=2, calls=1):
+    pr = gu.problem_of(w, rings=rings)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    ws = torch.empty(api.compass_workspace_bytes(pr, api.WS_PUSH), dtype=torch.uint8, device="cuda")
+    api.compass_workspace_init(ws)
+    # poison the gather buffers: a tile that reads rows before they arrive produces NaN
+    ws[api.STATUS_BYTES + 4096:].view(torch.int16).fill_(gu.NAN_BITS)
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    results = []
+    for _ in range(calls):
+        outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        api.compass_ag_gemm_push(pr, A, B, [o.view for o in outs], ws, torch.cuda.current_stream(), side)
+        status = api.compass_read_status(ws)
+        torch.cuda.synchronize()
+        assert status == (api.OK, 0)
+        assert all(o.guards_intact() for o in outs)
+        results.append([o.bits() for o in outs])
+    return results
+
+
+@pytest.mark.parametrize("P,m,N,K,rings", [
+    (1, 256, 256, 64, 2), (2, 256, 256, 256, 2), (2, 144, 264, 72, 2), (3, 272, 520, 344, 2), (4, 512, 768, 512, 2),
+    (4, 384, 1024, 320, 1), (8, 256, 512, 192, 2), (4, 1024, 2568, 200, 2),
+])
+def test_ag_gemm_push_small_shapes(P, m, N, K, rings):
+    w = small(wl.OP_AG_GEMM, P, m, N, K, dist=0.1)
+    A, B = wl.make_inputs(w)
+    (outs,) = run_push(w, A, B, rings=rings)
+    check_all(outs, ops.ag_gemm(A, B, rings=rings), w.name)
+
+
+def test_ag_gemm_push_repeated_calls_share_a_workspace():
+    w = small(wl.OP_AG_GEMM, 4, 512, 520, 200, dist=0.1)
+    A, B = wl.make_inputs(w)
+    first, second, third = run_push(w, A, B, calls=3)
+    ref = ops.ag_gemm(A, B)
+    for outs in (first, second, third):
+        check_all(outs, ref, w.name)
+
+
+def test_config2_ag_gemm_push_full_size_sampled():
+    w = wl.C2_AG
+    A, B = wl.make_inputs(w)
+    (outs,) = run_push(w, A, B)
+    rows = gu.sample_rows(w.M, w.P, 2)
+    refs = ops.ag_gemm(A, B, rows=rows)
+    for r in range(w.P):
+        assert not np.any((outs[r] & 0x7F80) == 0x7F80), "NaN/Inf or unwritten output"
+        rep = compare.check(outs[r][rows], refs[r])
+        assert rep.ok, f"{w.name} rank {r}: {rep}"
