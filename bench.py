@@ -36,8 +36,8 @@ UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes (read + written) per launch of the GEMM kernel from the ncu capture summarised in
-# profiles/gemm_mixed_kernel_C2_C3.md.
+# DRAM bytes (read + written) per launch of the GEMM kernel, from an ncu capture of
+# `bench.py --steps 1 --warmup 3 --no-cpu-baseline --no-sweep` (dram__bytes_read.sum + dram__bytes_write.sum).
 NCU_TRAFFIC_BYTES = {"C2": 359.1e6, "C3": 830.9e6}
 
 

@@ -86,6 +86,10 @@ enum { COMPASS_STRATEGY_INTRAFUSION = 0, COMPASS_STRATEGY_INTERDECOM = 1 };
  * need contributor s of a partition to precede contributor s+1 in the launch);
  * the segmented-K variant has one block per partition and ignores the field. */
 enum { COMPASS_ORDER_RANK_MAJOR = 0, COMPASS_ORDER_STEP_MAJOR = 1 };
+/* Sub-AllGather of compass_decomp: one gather kernel per stage (a single launch, as a library
+ * collective would be; it shares the SMs with the sub-GEMM it overlaps), or P*P device-to-device
+ * copies per stage on the copy engines (no SM use, but P*P*d calls on the host). */
+enum { COMPASS_COPY_KERNEL = 0, COMPASS_COPY_ENGINES = 1 };
 /* selectors for compass_workspace_bytes */
 enum { COMPASS_WS_FUSED = 0, COMPASS_WS_DECOMP = 1, COMPASS_WS_PUSH = 2 };
 
@@ -100,7 +104,7 @@ typedef struct compass_problem {
   int32_t dtype;       /* COMPASS_DTYPE_BF16 */
   int32_t rs_variant;  /* COMPASS_RS_* (GEMM+ReduceScatter only) */
   int32_t order;       /* COMPASS_ORDER_* : how the P logical ranks share the one GPU */
-  int32_t reserved;    /* must be 0 */
+  int32_t copy_mode;   /* COMPASS_COPY_* : how compass_decomp moves the AllGather slices */
 } compass_problem;
 
 /* One line of the ring chunk schedule (Section III-B).  `part` = rings*chunk +
@@ -199,9 +203,10 @@ int compass_gemm_rs(const compass_problem* problem, const void* const* A, const 
  * The same result as the fused calls, computed as problem->d sub-operators
  * pipelined on two streams.  The operator is split along rows: with
  * s = M/P/d, sub-operator j handles rows [j*s, (j+1)*s) of every chunk.
- *   AG: sub-collective j = device-to-device copies of row slice j of every
- *       shard into every rank's gather buffer (in the workspace) on
- *       stream_copy; sub-GEMM j on stream_compute once they have landed.
+ *   AG: sub-collective j = row slice j of every shard copied into every
+ *       rank's gather buffer (in the workspace) on stream_copy, by one gather
+ *       kernel or by copy-engine copies (problem->copy_mode); sub-GEMM j on
+ *       stream_compute once they have landed.
  *   RS: sub-GEMM j writes every rank's BF16 partial rows (workspace) on
  *       stream_compute; sub-collective j = a reduce kernel on stream_copy
  *       that sums the P partial slices in FP32 into the owners' rows.

@@ -23,6 +23,7 @@ DTYPE_BF16 = 0
 RS_SEGMENTED_K, RS_RING_RMW = 0, 1
 STRATEGY_INTRAFUSION, STRATEGY_INTERDECOM = 0, 1
 ORDER_RANK_MAJOR, ORDER_STEP_MAJOR = 0, 1
+COPY_KERNEL, COPY_ENGINES = 0, 1
 WS_FUSED, WS_DECOMP, WS_PUSH = 0, 1, 2
 MAX_P = 16
 STATUS_BYTES = 256
@@ -47,7 +48,7 @@ class CompassError(RuntimeError):
 class Problem(C.Structure):
     _fields_ = [("op", C.c_int32), ("P", C.c_int32), ("rings", C.c_int32), ("d", C.c_int32),
                 ("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64),
-                ("dtype", C.c_int32), ("rs_variant", C.c_int32), ("order", C.c_int32), ("reserved", C.c_int32)]
+                ("dtype", C.c_int32), ("rs_variant", C.c_int32), ("order", C.c_int32), ("copy_mode", C.c_int32)]
 
 
 class SchedEntry(C.Structure):
@@ -134,9 +135,10 @@ def _check(status: int, where: str) -> None:
 
 
 def make_problem(op: int, P: int, M: int, N: int, K: int, rings: int = 2, d: int = 1,
-                 rs_variant: int = RS_SEGMENTED_K, dtype: int = DTYPE_BF16, order: int = ORDER_RANK_MAJOR) -> Problem:
+                 rs_variant: int = RS_SEGMENTED_K, dtype: int = DTYPE_BF16, order: int = ORDER_RANK_MAJOR,
+                 copy_mode: int = COPY_KERNEL) -> Problem:
     return Problem(op=op, P=P, rings=rings, d=d, M=M, N=N, K=K, dtype=dtype, rs_variant=rs_variant, order=order,
-                   reserved=0)
+                   copy_mode=copy_mode)
 
 
 # ---- host-only calls -------------------------------------------------------------

@@ -25,8 +25,8 @@ int validate_problem(const compass_problem* pr, int want_op, bool need_d) {
   if (want_op >= 0 && pr->op != want_op) return COMPASS_ERR_INVALID_ARG;
   if (pr->P < 1 || (pr->rings != 1 && pr->rings != 2)) return COMPASS_ERR_INVALID_ARG;
   if (need_d && pr->d < 1) return COMPASS_ERR_INVALID_ARG;
-  if ((pr->order != COMPASS_ORDER_RANK_MAJOR && pr->order != COMPASS_ORDER_STEP_MAJOR) || pr->reserved != 0)
-    return COMPASS_ERR_INVALID_ARG;
+  if (pr->order != COMPASS_ORDER_RANK_MAJOR && pr->order != COMPASS_ORDER_STEP_MAJOR) return COMPASS_ERR_INVALID_ARG;
+  if (pr->copy_mode != COMPASS_COPY_KERNEL && pr->copy_mode != COMPASS_COPY_ENGINES) return COMPASS_ERR_INVALID_ARG;
   if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant != COMPASS_RS_SEGMENTED_K && pr->rs_variant != COMPASS_RS_RING_RMW)
     return COMPASS_ERR_INVALID_ARG;
   if (pr->dtype != COMPASS_DTYPE_BF16 || pr->P > COMPASS_MAX_P) return COMPASS_ERR_UNSUPPORTED;
@@ -282,13 +282,20 @@ int decomp_ag(const compass_problem* pr, const void* const* A, const void* const
   if ((e = cudaStreamWaitEvent(s_copy, ev[0], 0)) != cudaSuccess) return record_cuda_error(e);
   for (int j = 0; j < d; ++j) {
     // sub-AllGather j: row slice j of every shard into every rank's gather buffer
-    for (int r = 0; r < P; ++r)
-      for (int q = 0; q < P; ++q) {
-        const uint8_t* src = static_cast<const uint8_t*>(A[q]) + size_t(j * sl) * size_t(K) * 2;
-        uint8_t* dst = G[r] + size_t(q * m + j * sl) * size_t(K) * 2;
-        e = cudaMemcpyAsync(dst, src, size_t(sl) * size_t(K) * 2, cudaMemcpyDeviceToDevice, s_copy);
-        if (e != cudaSuccess) return record_cuda_error(e);
-      }
+    if (pr->copy_mode == COMPASS_COPY_ENGINES) {
+      for (int r = 0; r < P; ++r)
+        for (int q = 0; q < P; ++q) {
+          const uint8_t* src = static_cast<const uint8_t*>(A[q]) + size_t(j * sl) * size_t(K) * 2;
+          uint8_t* dst = G[r] + size_t(q * m + j * sl) * size_t(K) * 2;
+          e = cudaMemcpyAsync(dst, src, size_t(sl) * size_t(K) * 2, cudaMemcpyDeviceToDevice, s_copy);
+          if (e != cudaSuccess) return record_cuda_error(e);
+        }
+    } else {
+      void* gptr[kMaxP];
+      for (int r = 0; r < P; ++r) gptr[r] = G[r];
+      int stg = launch_gather_slices(A, gptr, P, m, K, j * sl, sl, s_copy);
+      if (stg != COMPASS_OK) return stg;
+    }
     if ((e = cudaEventRecord(ev[1 + j], s_copy)) != cudaSuccess) return record_cuda_error(e);
     if ((e = cudaStreamWaitEvent(s_comp, ev[1 + j], 0)) != cudaSuccess) return record_cuda_error(e);
     // sub-GEMM j on the gathered rows

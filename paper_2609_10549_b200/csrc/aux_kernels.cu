@@ -20,12 +20,14 @@ struct ReduceParams {
 };
 
 __device__ __forceinline__ void accumulate_bf16x8(float (&acc)[8], const uint4& v) {
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    acc[2 * i + 0] += __uint_as_float(w[i] << 16);
-    acc[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
-  }
+  acc[0] += __uint_as_float(v.x << 16);
+  acc[1] += __uint_as_float(v.x & 0xFFFF0000u);
+  acc[2] += __uint_as_float(v.y << 16);
+  acc[3] += __uint_as_float(v.y & 0xFFFF0000u);
+  acc[4] += __uint_as_float(v.z << 16);
+  acc[5] += __uint_as_float(v.z & 0xFFFF0000u);
+  acc[6] += __uint_as_float(v.w << 16);
+  acc[7] += __uint_as_float(v.w & 0xFFFF0000u);
 }
 
 __global__ void __launch_bounds__(256) reduce_partials_kernel(const __grid_constant__ ReduceParams p) {
@@ -48,7 +50,58 @@ __global__ void __launch_bounds__(256) reduce_partials_kernel(const __grid_const
   }
 }
 
+// Sub-AllGather of one InterDecom stage as ONE launch (what a library collective would be): row
+// slice [slice_begin, +slice_rows) of every shard goes to every rank's gather buffer.  Every
+// 16-byte vector is read once and written to the P destinations.
+struct GatherParams {
+  const uint4* shard[kMaxP];     // A_q [m x K]
+  uint4* gather[kMaxP];          // G_r [M x K]
+  int32_t P;
+  int64_t m;
+  int64_t k_vec;                 // K / 8
+  int64_t slice_begin, slice_rows;
+};
+
+__global__ void __launch_bounds__(256) gather_slices_kernel(const __grid_constant__ GatherParams p) {
+  const int64_t per_shard = p.slice_rows * p.k_vec;
+  const int64_t total = per_shard * p.P;
+  for (int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += int64_t(gridDim.x) * blockDim.x) {
+    const int q = int(i / per_shard);
+    const int64_t w = i - int64_t(q) * per_shard;
+    const uint4 v = __ldg(p.shard[q] + p.slice_begin * p.k_vec + w);
+    const int64_t dst = (int64_t(q) * p.m + p.slice_begin) * p.k_vec + w;
+    for (int r = 0; r < p.P; ++r) p.gather[r][dst] = v;
+  }
+}
+
 }  // namespace
+
+int launch_gather_slices(const void* const* shard, void* const* gather, int P, int64_t m, int64_t K, int64_t slice_begin,
+                         int64_t slice_rows, cudaStream_t stream) {
+  GatherParams p;
+  for (int q = 0; q < P; ++q) {
+    p.shard[q] = static_cast<const uint4*>(shard[q]);
+    p.gather[q] = static_cast<uint4*>(gather[q]);
+  }
+  p.P = P;
+  p.m = m;
+  p.k_vec = K / 8;
+  p.slice_begin = slice_begin;
+  p.slice_rows = slice_rows;
+  const int64_t total = slice_rows * p.k_vec * P;
+  if (total <= 0) return COMPASS_OK;
+  int dev = 0, num_sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return record_cuda_error(e);
+  e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return record_cuda_error(e);
+  const int64_t want = (total + 255) / 256, cap = int64_t(num_sms) * 4;
+  gather_slices_kernel<<<int(want < cap ? want : cap), 256, 0, stream>>>(p);
+  count_kernel_launch();
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return record_cuda_error(e);
+  return COMPASS_OK;
+}
 
 int launch_reduce_partials(const void* const* partial, int P, void* const* out, int64_t m, int64_t N, int64_t slice_begin,
                            int64_t slice_rows, cudaStream_t stream) {

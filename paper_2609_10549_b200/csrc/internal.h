@@ -137,6 +137,9 @@ int gemm_tile_rows(int mode, int rows_per_block);   // rows of one scheduling ti
 int launch_reduce_partials(const void* const* partial, int P, void* const* out, int64_t m, int64_t N,
                            int64_t slice_begin, int64_t slice_rows, cudaStream_t stream);
 
+int launch_gather_slices(const void* const* shard, void* const* gather, int P, int64_t m, int64_t K, int64_t slice_begin,
+                         int64_t slice_rows, cudaStream_t stream);
+
 // api.cu
 int record_cuda_error(cudaError_t e);
 void count_kernel_launch();

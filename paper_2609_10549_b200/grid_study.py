@@ -1,0 +1,215 @@
+"""Scores the performance models and the selector over the paper's parameter grid.
+
+Table IV spans hidden size K x intermediate size N x world size x sequence
+length M x pattern = 288 cases, with the decomposition degree swept inside
+each case.  For every case this script times, through the C ABI,
+
+  * the fused kernel (gather by address / segmented K),
+  * for AllGather+GEMM the readiness-driven variant (pushed partitions + flags),
+  * the decomposed pipeline for d in {1, 2, 4, 8, 16},
+
+then fits the models' parameters on half of the cases (Section IV-C: one-time
+offline regression) and scores them on the other half: mean absolute error of
+the decomposition model with and without the overhead factor (the comparison
+of Table II), of the fusion model with and without its overhead term, how often
+Eq. 4-5 pick the measured-best degree, what a fixed d = 4 costs, and how often
+Algorithm 1 picks the measured-faster strategy.
+
+Mapping of Table IV onto the two operators of one MLP block (Section II-A):
+AllGather+GEMM multiplies [M x K] by the column-parallel [K x N/P];
+GEMM+ReduceScatter multiplies [M x N/P] by the row-parallel [N/P x K].
+
+    python -m paper_2609_10549_b200.grid_study measure --out grid.jsonl [--shard i/n] [--max-m 32768]
+    python -m paper_2609_10549_b200.grid_study analyze --inp grid.jsonl
+
+`measure` appends one JSON line per case and skips cases already in the file.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import numpy as np
+
+from . import api
+from . import workloads as wl
+
+HIDDEN = (4096, 8192, 16384)
+INTER = (2048, 4096, 8192, 16384)
+WORLD = (4, 8)
+SEQ = (2048, 4096, 8192, 12288, 16384, 32768)
+DEGREES = (1, 2, 4, 8, 16)
+
+
+def grid(max_m=32768):
+    cases = []
+    for op in (wl.OP_AG_GEMM, wl.OP_GEMM_RS):
+        for P in WORLD:
+            for K in HIDDEN:
+                for N in INTER:
+                    for M in SEQ:
+                        if M > max_m:
+                            continue
+                        if op == wl.OP_AG_GEMM:
+                            shape = dict(op=op, P=P, M=M, N=N // P, K=K)
+                        else:
+                            shape = dict(op=op, P=P, M=M, N=K, K=N // P)
+                        cases.append(dict(shape, table_K=K, table_N=N))
+    return cases
+
+
+def case_key(c):
+    return f"{c['op']}-{c['P']}-{c['M']}-{c['table_N']}-{c['table_K']}"
+
+
+def measure(args):
+    import torch
+
+    done = set()
+    if os.path.exists(args.out):
+        with open(args.out) as f:
+            done = {case_key(json.loads(line)) for line in f if line.strip()}
+    cases = grid(args.max_m)
+    i, n = (int(x) for x in args.shard.split("/"))
+    cases = [c for k, c in enumerate(cases) if k % n == i]
+    stream = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+
+    def median_ms(fn, iters, warm=1):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(iters):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return float(np.median(ts))
+
+    for c in cases:
+        if case_key(c) in done:
+            continue
+        w = wl.Workload("grid", c["op"], P=c["P"], M=c["M"], N=c["N"], K=c["K"])
+        g = torch.Generator(device="cuda")
+        g.manual_seed(1)
+        mk = lambda shape, std: (torch.randn(shape, device="cuda", dtype=torch.float32, generator=g) * std).to(torch.bfloat16)
+        A = [mk(w.a_shape, 1.0) for _ in range(w.P)]
+        B = [mk(w.b_shape, 0.02) for _ in range(w.P)]
+        out = [torch.empty(w.out_shape, dtype=torch.bfloat16, device="cuda") for _ in range(w.P)]
+        pr = api.make_problem(w.op, w.P, w.M, w.N, w.K)
+        ws = api.alloc_workspace(pr)
+        iters = 5
+        fused = api.compass_ag_gemm if w.op == wl.OP_AG_GEMM else api.compass_gemm_rs
+        rec = dict(c, flops=w.flops, m_rows=w.m)
+        rec["fused_ms"] = median_ms(lambda: fused(pr, A, B, out, ws, stream), iters)
+        if w.op == wl.OP_AG_GEMM:
+            pws = torch.empty(api.compass_workspace_bytes(pr, api.WS_PUSH), dtype=torch.uint8, device="cuda")
+            api.compass_workspace_init(pws)
+            rec["push_ms"] = median_ms(lambda: api.compass_ag_gemm_push(pr, A, B, out, pws, stream, side), iters)
+            del pws
+        dws = None
+        rec["decomp_ms"] = {}
+        for d in DEGREES:
+            if w.m % d:
+                continue
+            prd = api.make_problem(w.op, w.P, w.M, w.N, w.K, d=d)
+            if dws is None:
+                dws = api.alloc_workspace(prd, api.WS_DECOMP)
+            rec["decomp_ms"][str(d)] = median_ms(lambda: api.compass_decomp(prd, A, B, out, dws, stream, side), iters)
+        status = api.compass_read_status(ws)
+        if status != (api.OK, 0):
+            raise SystemExit(f"device status {status} on {c}")
+        with open(args.out, "a") as f:
+            f.write(json.dumps(rec) + "\n")
+        print(case_key(c), round(rec["fused_ms"], 3), {k: round(v, 3) for k, v in rec["decomp_ms"].items()}, flush=True)
+        del A, B, out, ws, dws
+        torch.cuda.empty_cache()
+
+
+def analyze(args):
+    with open(args.inp) as f:
+        recs = [json.loads(line) for line in f if line.strip()]
+    report = {"cases": len(recs)}
+    for op, name in ((wl.OP_AG_GEMM, "AG+GEMM"), (wl.OP_GEMM_RS, "GEMM+RS")):
+        rs = sorted((r for r in recs if r["op"] == op), key=case_key)
+        if len(rs) < 4:
+            continue
+        for r in rs:
+            r["t_comp"] = r["fused_ms"]                                      # same FLOPs, no sub-collective
+            r["t_comm"] = max(r["decomp_ms"]["1"] - r["fused_ms"], 1e-4)     # T(1) = T_comp + T_comm
+            r["t_intra"] = r.get("push_ms") or r["fused_ms"]
+            r["volume"] = float(r["M"]) * (r["K"] if op == wl.OP_AG_GEMM else r["N"])
+            r["bytes"] = 2.0 * r["P"] * r["volume"]
+        cal, test = rs[0::2], rs[1::2]
+        ca, cb = api.compass_calib_fit_line([r["flops"] for r in cal], [r["t_comp"] for r in cal])
+        ma, mb = api.compass_calib_fit_line([r["bytes"] for r in cal], [r["t_comm"] for r in cal])
+        tc, tm, dd, tt = [], [], [], []
+        for r in cal:
+            for d, t in r["decomp_ms"].items():
+                if int(d) > 1:
+                    tc.append(r["t_comp"]); tm.append(r["t_comm"]); dd.append(int(d)); tt.append(t)
+        alpha, beta = api.compass_calib_fit_decomp(tc, tm, dd, tt)
+        af, bf = api.compass_calib_fit_fusion([r["t_comp"] for r in cal], [r["t_comm"] for r in cal], [r["P"] for r in cal],
+                                              [r["volume"] for r in cal], [r["t_intra"] for r in cal])
+        calib = api.Calib(ca, cb, ma, mb, alpha, beta, af, bf)
+        mae_aware = {d: [] for d in DEGREES[1:]}
+        mae_agn = {d: [] for d in DEGREES[1:]}
+        fus_aware, fus_agn, d_hits, strat_hits, fixed4_penalty, pred_penalty = [], [], [], [], [], []
+        best_hist = {}
+        for r in test:
+            for d in DEGREES[1:]:
+                if str(d) in r["decomp_ms"]:
+                    meas = r["decomp_ms"][str(d)]
+                    mae_aware[d].append(abs(api.compass_model_decomp_time(r["t_comp"], r["t_comm"], alpha, beta, d) - meas))
+                    mae_agn[d].append(abs(api.compass_model_decomp_time(r["t_comp"], r["t_comm"], 1.0, 0.0, d) - meas))
+            fus_aware.append(abs(api.compass_model_fusion_time(r["t_comp"], r["t_comm"], r["P"], af, bf, r["volume"]) - r["t_intra"]))
+            fus_agn.append(abs(api.compass_model_fusion_time(r["t_comp"], r["t_comm"], r["P"], 0.0, 0.0, r["volume"]) - r["t_intra"]))
+            best_d = min(r["decomp_ms"], key=lambda k: r["decomp_ms"][k])
+            best_hist[best_d] = best_hist.get(best_d, 0) + 1
+            choice = api.compass_select(api.make_problem(op, r["P"], r["M"], r["N"], r["K"]), calib)
+            d_hits.append(int(str(choice.d_star) == best_d))
+            t_best = r["decomp_ms"][best_d]
+            pred_penalty.append(r["decomp_ms"].get(str(choice.d_star), t_best) / t_best - 1.0)
+            if "4" in r["decomp_ms"]:
+                fixed4_penalty.append(r["decomp_ms"]["4"] / t_best - 1.0)
+            winner = api.STRATEGY_INTRAFUSION if r["t_intra"] < t_best else api.STRATEGY_INTERDECOM
+            strat_hits.append(int(choice.strategy == winner))
+        mean = lambda xs: float(np.mean(xs)) if xs else None
+        report[name] = {
+            "calibration_cases": len(cal), "test_cases": len(test),
+            "calib": {"comp_a": ca, "comp_b": cb, "comm_a": ma, "comm_b": mb, "alpha_decomp": alpha, "beta_decomp": beta,
+                      "alpha_fusion": af, "beta_fusion": bf},
+            "decomp_mae_ms_overhead_aware": {str(d): mean(v) for d, v in mae_aware.items()},
+            "decomp_mae_ms_overhead_agnostic": {str(d): mean(v) for d, v in mae_agn.items()},
+            "decomp_mae_ms_overall": {"aware": mean(sum(mae_aware.values(), [])), "agnostic": mean(sum(mae_agn.values(), []))},
+            "mean_decomp_time_ms": mean([t for r in test for t in r["decomp_ms"].values()]),
+            "fusion_mae_ms": {"aware": mean(fus_aware), "agnostic": mean(fus_agn)},
+            "measured_best_d_histogram": best_hist,
+            "predicted_d_is_best": mean(d_hits),
+            "penalty_of_predicted_d": mean(pred_penalty), "penalty_of_fixed_d4": mean(fixed4_penalty),
+            "selector_accuracy": mean(strat_hits),
+            "intrafusion_wins": int(sum(1 for r in test if r["t_intra"] < min(r["decomp_ms"].values()))),
+        }
+    print(json.dumps(report, indent=1))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    sub = ap.add_subparsers(dest="cmd", required=True)
+    m = sub.add_parser("measure")
+    m.add_argument("--out", required=True)
+    m.add_argument("--shard", default="0/1")
+    m.add_argument("--max-m", type=int, default=32768)
+    a = sub.add_parser("analyze")
+    a.add_argument("--inp", required=True)
+    args = ap.parse_args()
+    (measure if args.cmd == "measure" else analyze)(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -38,8 +38,8 @@ def device_inputs(A_bits, B_bits):
     return [api.to_device(a) for a in A_bits], [api.to_device(b) for b in B_bits]
 
 
-def problem_of(w: wl.Workload, rings=2, d=1, rs_variant=api.RS_SEGMENTED_K) -> api.Problem:
-    return api.make_problem(w.op, w.P, w.M, w.N, w.K, rings=rings, d=d, rs_variant=rs_variant)
+def problem_of(w: wl.Workload, rings=2, d=1, rs_variant=api.RS_SEGMENTED_K, copy_mode=api.COPY_KERNEL) -> api.Problem:
+    return api.make_problem(w.op, w.P, w.M, w.N, w.K, rings=rings, d=d, rs_variant=rs_variant, copy_mode=copy_mode)
 
 
 def run_fused(w: wl.Workload, A_bits, B_bits, rings=2, rs_variant=api.RS_SEGMENTED_K):
@@ -57,8 +57,8 @@ def run_fused(w: wl.Workload, A_bits, B_bits, rings=2, rs_variant=api.RS_SEGMENT
     return [o.bits() for o in outs], (status, detail), all(o.guards_intact() for o in outs)
 
 
-def run_decomp(w: wl.Workload, A_bits, B_bits, d: int, two_streams=True):
-    pr = problem_of(w, d=d)
+def run_decomp(w: wl.Workload, A_bits, B_bits, d: int, two_streams=True, copy_mode=api.COPY_KERNEL):
+    pr = problem_of(w, d=d, copy_mode=copy_mode)
     A, B = device_inputs(A_bits, B_bits)
     outs = [Guarded(*w.out_shape) for _ in range(w.P)]
     ws = api.alloc_workspace(pr, api.WS_DECOMP)

@@ -169,8 +169,7 @@ def test_problem_validation_codes():
     rs = api.make_problem(OP_GEMM_RS, 8, 8192, 4096, 1376, rs_variant=5)
     assert _codes(rs)[0] == api.ERR_INVALID_ARG
     assert _codes(api.make_problem(**ok, order=2))[0] == api.ERR_INVALID_ARG
-    res = api.make_problem(**ok); res.reserved = 1
-    assert _codes(res)[0] == api.ERR_INVALID_ARG
+    assert _codes(api.make_problem(**ok, copy_mode=2))[0] == api.ERR_INVALID_ARG
 
 
 def test_workspace_sizes():

@@ -175,10 +175,11 @@ def test_config5_gemm_rs_full_size_sampled():
 def test_interdecom_small_shapes(op, P, m, N, K, d):
     w = small(op, P, m, N, K, dist=0.1)
     A, B = wl.make_inputs(w)
-    outs, status, guards = gu.run_decomp(w, A, B, d)
-    assert status == (api.OK, 0) and guards
     refs = ops.decomp_ag_gemm(A, B, d) if op == wl.OP_AG_GEMM else ops.decomp_gemm_rs(A, B, d)
-    check_all(outs, refs, f"{w.name} d={d}")
+    for copy_mode in ((api.COPY_KERNEL, api.COPY_ENGINES) if op == wl.OP_AG_GEMM else (api.COPY_KERNEL,)):
+        outs, status, guards = gu.run_decomp(w, A, B, d, copy_mode=copy_mode)
+        assert status == (api.OK, 0) and guards
+        check_all(outs, refs, f"{w.name} d={d} copy_mode={copy_mode}")
 
 
 @pytest.mark.parametrize("d", [1, 4, 16])
