@@ -212,7 +212,7 @@ def workload_config(w_ag, w_rs):
 # ---------------------------------------------------------------------------------
 # InterDecom sweep, calibration of the models, strategy selection (reported beside the headline number)
 
-def interdecom_report(torch, api):
+def interdecom_report(torch, api, hbm_gbs):
     """Times compass_decomp for d in {1,2,4,8,16} on the config-4 shapes, fits
     the models' parameters on other shapes (Section IV-C: one-time offline
     regression), and sets the measured-best degree and strategy beside the
@@ -311,7 +311,19 @@ def interdecom_report(torch, api):
         # IntraFusion as the paper builds it moves the partitions while it computes: compare that variant with
         # InterDecom where it exists; the gather-by-address kernel (no transfers at all) is reported beside it.
         t_intra = t_push if t_push is not None else t_fused
+        # HBM-bound phase of the sequential (d = 1) run, which does not overlap it with the GEMM: the gather
+        # kernel reads every shard once and writes it to the P gather buffers; the reduce kernel reads the P
+        # BF16 partials and writes the owners' rows.
+        if w.op == wl.OP_AG_GEMM:
+            phase, phase_bytes = "gather", 2.0 * w.M * w.K * (1 + w.P)
+        else:
+            phase, phase_bytes = "reduce", 2.0 * w.M * w.N * (w.P + 1)
+        phase_ms = max(times[1] - t_fused, 1e-6)
         out = {"workload": w.name, "fused_ms": t_fused, "push_ms": t_push,
+               "hbm_phase": {"kernel": phase, "ms": phase_ms, "algorithmic_bytes": phase_bytes,
+                             "gbs": phase_bytes / (phase_ms * 1e-3) / 1e9,
+                             "frac_of_measured_hbm": phase_bytes / (phase_ms * 1e-3) / 1e9 / hbm_gbs,
+                             "how": "T_decomp(d=1) - T_fused: the phase runs strictly before (gather) or after (reduce) the GEMM"},
                "decomp_ms": {str(d): t for d, t in times.items()},
                "measured_best_d": best_d, "predicted_d": choice.d_star,
                "predicted_strategy": "IntraFusion" if choice.strategy == api.STRATEGY_INTRAFUSION else "InterDecom",
@@ -525,7 +537,7 @@ def run_ours(args, w_ag, w_rs):
         if world == 1 and not args.no_sweep:
             del hag, hrs
             torch.cuda.empty_cache()
-            line["interdecom"] = interdecom_report(torch, api)
+            line["interdecom"] = interdecom_report(torch, api, peaks["hbm_gbs"])
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w_ag, w_rs)
         print(json.dumps(line), flush=True)

@@ -40,7 +40,11 @@ __global__ void __launch_bounds__(256) reduce_partials_kernel(const __grid_const
     const int64_t col = w - row * p.n_vec;
     const int64_t src = (int64_t(c) * p.m + p.slice_begin + row) * p.n_vec + col;
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    for (int q = 0; q < p.P; ++q) accumulate_bf16x8(acc, __ldg(p.partial[q] + src));
+#pragma unroll 1
+    for (int q = 0; q < p.P; ++q) {
+      const uint4 v = __ldg(p.partial[q] + src);
+      accumulate_bf16x8(acc, v);
+    }
     uint4 r;
     r.x = ptx::pack_bf16x2(acc[0], acc[1]);
     r.y = ptx::pack_bf16x2(acc[2], acc[3]);

@@ -421,42 +421,54 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
           if (!ready) break;
         }
       }
-      for (int c = 0; c < nchunks; ++c) {
-        uint32_t v[32];
-        tmem_ld_32x32b_x32(taddr + c * 32, v);
-        tmem_ld_wait();
-        if (c == nchunks - 1) {
-          // accumulator fully copied to registers: hand it back to the MMA issuer
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) {
-            if (kPair) mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->acc_empty[buf]), 0));
-            else mbar_arrive(&ctl->acc_empty[buf]);
+      // The running sum of this lane's row is fetched in one go, before the accumulator is read:
+      // the read-modify-write then pays one L2 round trip per tile instead of one per chunk.
+      uint4 prev[BN / 8];
+      if (add_previous && row_ok) {
+#pragma unroll
+        for (int g = 0; g < BN / 8; ++g)
+          if (g * 8 < ncols) prev[g] = __ldcg(reinterpret_cast<const uint4*>(orow + g * 8));   // written by another SM: from L2
+      }
+#pragma unroll
+      for (int c = 0; c < BN / 32; ++c) {
+        if (c < nchunks) {
+          uint32_t v[32];
+          tmem_ld_32x32b_x32(taddr + c * 32, v);
+          tmem_ld_wait();
+          if (c == nchunks - 1) {
+            // accumulator fully copied to registers: hand it back to the MMA issuer
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+              if (kPair) mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->acc_empty[buf]), 0));
+              else mbar_arrive(&ctl->acc_empty[buf]);
+            }
           }
-        }
-        if (row_ok) {
+          if (row_ok) {
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            if (c * 32 + g * 8 < ncols) {
-              uint4* dst = reinterpret_cast<uint4*>(orow + c * 32 + g * 8);
-              float f[8];
+            for (int g = 0; g < 4; ++g) {
+              if (c * 32 + g * 8 < ncols) {
+                float f[8];
 #pragma unroll
-              for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[g * 8 + i]);
-              if (add_previous) {
-                const uint4 old = __ldcg(dst);          // written by another SM: read it from L2
-                const uint32_t w[4] = {old.x, old.y, old.z, old.w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  f[2 * i + 0] += __uint_as_float(w[i] << 16);
-                  f[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
+                for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[g * 8 + i]);
+                if (add_previous) {
+                  const uint4 o = prev[c * 4 + g];
+                  f[0] += __uint_as_float(o.x << 16);
+                  f[1] += __uint_as_float(o.x & 0xFFFF0000u);
+                  f[2] += __uint_as_float(o.y << 16);
+                  f[3] += __uint_as_float(o.y & 0xFFFF0000u);
+                  f[4] += __uint_as_float(o.z << 16);
+                  f[5] += __uint_as_float(o.z & 0xFFFF0000u);
+                  f[6] += __uint_as_float(o.w << 16);
+                  f[7] += __uint_as_float(o.w & 0xFFFF0000u);
                 }
+                uint4 q;
+                q.x = pack_bf16x2(f[0], f[1]);
+                q.y = pack_bf16x2(f[2], f[3]);
+                q.z = pack_bf16x2(f[4], f[5]);
+                q.w = pack_bf16x2(f[6], f[7]);
+                *reinterpret_cast<uint4*>(orow + c * 32 + g * 8) = q;
               }
-              uint4 q;
-              q.x = pack_bf16x2(f[0], f[1]);
-              q.y = pack_bf16x2(f[2], f[3]);
-              q.z = pack_bf16x2(f[4], f[5]);
-              q.w = pack_bf16x2(f[6], f[7]);
-              *dst = q;
             }
           }
         }

@@ -352,3 +352,41 @@ def test_config2_ag_gemm_push_full_size_sampled():
         assert not np.any((outs[r] & 0x7F80) == 0x7F80), "NaN/Inf or unwritten output"
         rep = compare.check(outs[r][rows], refs[r])
         assert rep.ok, f"{w.name} rank {r}: {rep}"
+
+
+# ---- invariances: the same arithmetic in the same k order must give the same bits ------------------
+
+def test_launch_order_push_and_decomposition_do_not_change_a_bit():
+    """AllGather+GEMM sums every output element over k in the same order whatever the launch order,
+    whether the A rows are read in place or from a pushed copy, and however many row slices
+    InterDecom cuts: the BF16 outputs must be identical bit for bit."""
+    w = small(wl.OP_AG_GEMM, 4, 1024, 776, 328, dist=0.1)
+    A_bits, B_bits = wl.make_inputs(w)
+    A, B = gu.device_inputs(A_bits, B_bits)
+
+    def fused(order):
+        pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, order=order)
+        outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        ws = api.alloc_workspace(pr)
+        api.compass_ag_gemm(pr, A, B, [o.view for o in outs], ws)
+        assert api.compass_read_status(ws) == (api.OK, 0)
+        return [o.bits() for o in outs]
+
+    base = fused(api.ORDER_RANK_MAJOR)
+    others = {"step-major": fused(api.ORDER_STEP_MAJOR), "push": run_push(w, A_bits, B_bits)[0]}
+    for d in (1, 2, 8):
+        outs, status, guards = gu.run_decomp(w, A_bits, B_bits, d)
+        assert status == (api.OK, 0) and guards
+        others[f"decomp d={d}"] = outs
+    for name, outs in others.items():
+        for r in range(w.P):
+            assert np.array_equal(outs[r], base[r]), f"{name}: rank {r} differs"
+
+
+def test_single_ring_and_double_ring_agree_bitwise_for_ag_gemm():
+    w = small(wl.OP_AG_GEMM, 4, 512, 520, 200, dist=0.1)
+    A, B = wl.make_inputs(w)
+    two, _, _ = gu.run_fused(w, A, B, rings=2)
+    one, _, _ = gu.run_fused(w, A, B, rings=1)
+    for x, y in zip(one, two):
+        assert np.array_equal(x, y)
