@@ -144,7 +144,8 @@ typedef struct compass_plan_block {
   int32_t a_tensor, a_row_begin;       /* which A pointer is read, first row inside it */
   int32_t out_tensor, out_row_begin;   /* which output pointer is written, first row inside it */
   int32_t rows;
-  int32_t first_tile, tile_count;      /* tiles [first_tile, first_tile+tile_count) of the launch */
+  int32_t first_tile, tile_count;      /* position in the launch, counted in 256x256 output tiles (128x256 for blocks of
+                                          fewer than 256 rows); a 512x256 tile of the kernel counts as two */
 } compass_plan_block;
 
 /* ---- schedule (Section III-A, III-B) -------------------------------------
