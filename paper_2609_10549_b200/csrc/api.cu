@@ -237,16 +237,25 @@ int fused_call(const compass_problem* pr, int op, const void* const* A, const vo
 
 // ---- InterDecom ----------------------------------------------------------------
 
+// Events that order the two streams of a call; created on first use, one set per device
+// (an event belongs to the device that was current when it was created).
 struct EventPool {
+  static constexpr int kMaxDevices = 64;
   std::mutex mu;
-  cudaEvent_t ev[2 * 16 + 2];
-  int made = 0;
+  cudaEvent_t all[kMaxDevices][2 * 16 + 2];
+  int made[kMaxDevices] = {};
+  cudaEvent_t* ev = nullptr;      // the current device's set, valid after ensure()
   int ensure(int n) {
-    while (made < n) {
-      cudaError_t e = cudaEventCreateWithFlags(&ev[made], cudaEventDisableTiming);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (dev < 0 || dev >= kMaxDevices) return COMPASS_ERR_UNSUPPORTED;
+    while (made[dev] < n) {
+      e = cudaEventCreateWithFlags(&all[dev][made[dev]], cudaEventDisableTiming);
       if (e != cudaSuccess) return record_cuda_error(e);
-      ++made;
+      ++made[dev];
     }
+    ev = all[dev];
     return COMPASS_OK;
   }
 };

@@ -30,6 +30,8 @@
 // warp 1 = tensor-memory allocation + MMA issue (one lane), warps 2..5 =
 // epilogue (warp w reads TMEM lanes 32*(w%4)..+31).  Every wait is bounded and
 // reports COMPASS_ERR_TIMEOUT instead of hanging.
+#include <mutex>
+
 #include "internal.h"
 #include "ptx_sm100.cuh"
 
@@ -898,12 +900,19 @@ struct DeviceInfo {
   bool ready = false;
 };
 
+// Per-device facts, gathered the first time a device launches (function attributes and cluster
+// occupancy belong to the device that is current).
 int device_info(DeviceInfo** out) {
-  static DeviceInfo info;
+  constexpr int kMaxDevices = 64;
+  static DeviceInfo infos[kMaxDevices];
+  static std::mutex mu;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return record_cuda_error(e);
+  if (dev < 0 || dev >= kMaxDevices) return COMPASS_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(mu);
+  DeviceInfo& info = infos[dev];
   if (!info.ready) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return record_cuda_error(e);
     e = cudaDeviceGetAttribute(&info.num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return record_cuda_error(e);
     e = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<false>()));
