@@ -258,6 +258,14 @@ int compass_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_s
  * workspace (COMPASS_OK or COMPASS_ERR_TIMEOUT); *detail (may be NULL) gets
  * a code telling which wait gave up. */
 int compass_read_status(void* workspace, void* cuda_stream, int* detail);
+/* Synchronise the stream and return how long CTA 0 of the last GEMM kernel
+ * that used this workspace ran, in SM clock cycles and in nanoseconds (host
+ * pointers, both required).  cycles / nanoseconds is the SM clock the kernel
+ * really had: under the board's power cap a tensor-core kernel runs well
+ * below the nominal clock, and a throughput figure can only be judged against
+ * the clock it was obtained at.  A measurement aid, not part of the paper's
+ * method; both values are 0 before the first launch. */
+int compass_read_kernel_clock(void* workspace, void* cuda_stream, uint64_t* sm_cycles, uint64_t* nanoseconds);
 /* The blocks of the fused launch for this problem, in launch order. */
 int compass_launch_plan(const compass_problem* problem, compass_plan_block* out, size_t capacity, size_t* count);
 /* End-to-end convenience with HOST tensors: copies A and B (host pointers,

@@ -35,7 +35,7 @@ EXPORTS = (
     "compass_calib_fit_decomp", "compass_calib_fit_fusion", "compass_workspace_bytes", "compass_workspace_init",
     "compass_read_status", "compass_launch_plan", "compass_fused_host", "compass_status_string",
     "compass_last_cuda_error", "compass_kernel_launch_count", "compass_gemm_rs_sequential_noalloc",
-    "compass_set_wait_limit_us", "compass_calib_fit_line", "compass_ag_gemm_push",
+    "compass_set_wait_limit_us", "compass_calib_fit_line", "compass_ag_gemm_push", "compass_read_kernel_clock",
 )
 
 
@@ -100,6 +100,7 @@ def lib() -> C.CDLL:
         L.compass_workspace_bytes.argtypes = [C.POINTER(Problem), C.c_int, C.POINTER(C.c_size_t)]
         L.compass_workspace_init.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
         L.compass_read_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]
+        L.compass_read_kernel_clock.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
         L.compass_launch_plan.argtypes = [C.POINTER(Problem), C.POINTER(PlanBlock), C.c_size_t, C.POINTER(C.c_size_t)]
         L.compass_fused_host.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t),
                                          C.c_void_p, C.c_size_t, C.c_void_p]
@@ -250,6 +251,15 @@ def compass_read_status(workspace, stream=None):
     p, _ = _ws(workspace)
     st = lib().compass_read_status(p, _stream_handle(stream), C.byref(detail))
     return int(st), int(detail.value)
+
+
+def compass_read_kernel_clock(workspace, stream=None):
+    """(SM cycles, nanoseconds) of CTA 0 of the last GEMM kernel that used this workspace."""
+    cycles, ns = C.c_uint64(0), C.c_uint64(0)
+    p, _ = _ws(workspace)
+    _check(lib().compass_read_kernel_clock(p, _stream_handle(stream), C.byref(cycles), C.byref(ns)),
+           "compass_read_kernel_clock")
+    return int(cycles.value), int(ns.value)
 
 
 def compass_ag_gemm(problem: Problem, A: Sequence, B: Sequence, Cout: Sequence, workspace, stream=None) -> None:

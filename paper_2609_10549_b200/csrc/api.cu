@@ -431,6 +431,18 @@ extern "C" int compass_read_status(void* ws, void* stream, int* detail) {
   return host.code;
 }
 
+extern "C" int compass_read_kernel_clock(void* ws, void* stream, uint64_t* sm_cycles, uint64_t* nanoseconds) {
+  if (ws == nullptr || sm_cycles == nullptr || nanoseconds == nullptr) return COMPASS_ERR_INVALID_ARG;
+  StatusBlock host;
+  cudaError_t e = cudaMemcpyAsync(&host, ws, sizeof(host), cudaMemcpyDeviceToHost, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return record_cuda_error(e);
+  e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return record_cuda_error(e);
+  *sm_cycles = host.kernel_cycles;
+  *nanoseconds = host.kernel_ns;
+  return COMPASS_OK;
+}
+
 extern "C" int compass_launch_plan(const compass_problem* pr, compass_plan_block* out, size_t capacity, size_t* count) {
   if (count == nullptr) return COMPASS_ERR_INVALID_ARG;
   int st = validate_problem(pr, -1, false);

@@ -90,6 +90,25 @@ __device__ __forceinline__ void report_timeout(const GemmParams& p, Control* ctl
   }
 }
 
+// CTA 0 records how many SM cycles and nanoseconds it ran: their ratio is the clock the
+// kernel really had (under a power cap well below the nominal one).
+struct ClockRecord {
+  long long c0;
+  uint64_t t0;
+  __device__ __forceinline__ void begin() {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      c0 = clock64();
+      t0 = globaltimer_ns();
+    }
+  }
+  __device__ __forceinline__ void end(const GemmParams& p) const {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      p.status->kernel_cycles = static_cast<unsigned long long>(clock64() - c0);
+      p.status->kernel_ns = globaltimer_ns() - t0;
+    }
+  }
+};
+
 // Wait for an mbarrier phase, giving up after p.wait_limit_us or when another
 // role of this CTA has already given up.
 __device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, Control* ctl, const GemmParams& p, int site,
@@ -209,6 +228,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
   // work units: clusters in pair mode, CTAs otherwise
   const int unit = kPair ? int(blockIdx.x >> 1) : int(blockIdx.x);
   const int n_units = kPair ? int(gridDim.x >> 1) : int(gridDim.x);
+  ClockRecord clock_record;
+  clock_record.begin();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
@@ -499,6 +520,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     if (kPair) tmem_dealloc_pair(tmem_base, kTmemCols);
     else tmem_dealloc(tmem_base, kTmemCols);
   }
+  clock_record.end(p);
 }
 
 // ---- mixed-tile pair kernel ---------------------------------------------------------
@@ -607,6 +629,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
   const bool leader = cta_rank == 0;
   const int unit = int(blockIdx.x >> 1);
   const int n_units = int(gridDim.x >> 1);
+  ClockRecord clock_record;
+  clock_record.begin();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSlots; ++s) {
@@ -702,39 +726,106 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
         const uint32_t buf = big ? 0u : (small_rr & 1u);
         // the accumulator(s) this tile writes must have been drained by the epilogue
         if (!wait_bounded(&ctl->acc_empty[buf], ((buf ? uses1 : uses0) & 1u) ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
-        if (big && !wait_bounded(&ctl->acc_empty[1], (uses1 & 1u) ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
         tc_fence_after_sync();
-        const uint32_t acc_a = tmem_base + buf * BN;
-        int kb_in_seg = 0;
-        for (int kb = 0; kb < n_kb; ++kb, ++j) {
-          if (!wait_bounded(&ctl->full[j & 3u], (j >> 2) & 1u, ctl, p, WAIT_SMEM_FULL, t)) {
-            ok = false;
-            break;
+        if (big) {
+          // 512x256 tile: A block 0 -> accumulator 0, A block 1 -> accumulator 1, both with the stage's B chunk.
+          // In the body of the tile the two MMAs of a k-step are adjacent so that they read the same B slice
+          // back to back.  Both accumulators are live for the whole tile, so nothing hides the epilogue
+          // unless the two are skewed at the tile's ends: for the first and the last `skew` stages all of
+          // accumulator 0's MMAs are issued before accumulator 1's.  Accumulator 0 is then complete `skew`
+          // half-stages before the tile ends (the epilogue reads it while accumulator 1 finishes) and the
+          // next tile starts on it while the epilogue still drains accumulator 1.
+          const int skew = (n_kb >= 2 * p.skew) ? p.skew : 0;
+          auto ksteps = [&](int kb) { return (kb % kb_seg == kb_seg - 1) ? tail : BK / UMMA_K; };
+          auto issue = [&](uint32_t acc, int a_chunk, int b_chunk, int nk, uint32_t first) {
+            const uint64_t da = desc0 + uint64_t(((a_chunk % kChunks) * kChunkBytes) >> 4);
+            const uint64_t db = desc0 + uint64_t(((b_chunk % kChunks) * kChunkBytes) >> 4);
+            if (nk == BK / UMMA_K) {
+#pragma unroll
+              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc, da + uint64_t(k * 2), db + uint64_t(k * 2), idesc, k ? 1u : first);
+            } else {
+              for (int k = 0; k < nk; ++k) umma_bf16_pair(acc, da + uint64_t(k * 2), db + uint64_t(k * 2), idesc, k ? 1u : first);
+            }
+          };
+          // `count` stages from stage kb on, accumulator 0 first, then accumulator 1 (which releases the stages)
+          auto skewed = [&](int kb, int count, bool wait_acc1) -> bool {
+            for (int s = 0; s < count; ++s) {
+              if (!wait_bounded(&ctl->full[(j + s) & 3u], ((j + s) >> 2) & 1u, ctl, p, WAIT_SMEM_FULL, t)) return false;
+              tc_fence_after_sync();
+              issue(tmem_base, chunk + 3 * s, chunk + 3 * s + 2, ksteps(kb + s), (kb + s) != 0 ? 1u : 0u);
+            }
+            if (wait_acc1) {
+              if (!wait_bounded(&ctl->acc_empty[1], (uses1 & 1u) ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) return false;
+              tc_fence_after_sync();
+            } else {
+              umma_commit_pair(&ctl->acc_full[0], 0x3);
+            }
+            for (int s = 0; s < count; ++s) {
+              issue(tmem_base + BN, chunk + 3 * s + 1, chunk + 3 * s + 2, ksteps(kb + s), (kb + s) != 0 ? 1u : 0u);
+              umma_commit_pair(&ctl->empty[(j + s) & 3u], 0x3);
+            }
+            j += uint32_t(count);
+            chunk = (chunk + 3 * count) % kChunks;
+            return true;
+          };
+          int kb = 0;
+          if (skew) {
+            if (!skewed(0, skew, true)) { ok = false; break; }
+            kb = skew;
+          } else {
+            if (!wait_bounded(&ctl->acc_empty[1], (uses1 & 1u) ^ 1u, ctl, p, WAIT_ACC_EMPTY, t)) break;
+            tc_fence_after_sync();
           }
-          tc_fence_after_sync();
-          const bool full_stage = kb_in_seg != kb_seg - 1 || tail == 2 * BK / UMMA_K || (big && tail == BK / UMMA_K);
-          const uint64_t d0 = desc0 + uint64_t((((chunk + 0) % kChunks) * kChunkBytes) >> 4);
-          const uint64_t d1 = desc0 + uint64_t((((chunk + 1) % kChunks) * kChunkBytes) >> 4);
-          const uint64_t d2 = desc0 + uint64_t((((chunk + 2) % kChunks) * kChunkBytes) >> 4);
-          const uint32_t first = kb != 0 ? 1u : 0u;
-          if (big) {
-            // A block 0 -> accumulator 0, A block 1 -> accumulator 1.  The two MMAs of a
-            // k-step are adjacent so that they read the same B slice back to back.
-            if (full_stage) {
+          for (; kb < n_kb - skew; ++kb, ++j) {
+            if (!wait_bounded(&ctl->full[j & 3u], (j >> 2) & 1u, ctl, p, WAIT_SMEM_FULL, t)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after_sync();
+            const uint64_t d0 = desc0 + uint64_t((((chunk + 0) % kChunks) * kChunkBytes) >> 4);
+            const uint64_t d1 = desc0 + uint64_t((((chunk + 1) % kChunks) * kChunkBytes) >> 4);
+            const uint64_t d2 = desc0 + uint64_t((((chunk + 2) % kChunks) * kChunkBytes) >> 4);
+            const uint32_t first = kb != 0 ? 1u : 0u;
+            const int nk = ksteps(kb);
+            if (nk == BK / UMMA_K) {
 #pragma unroll
               for (int k = 0; k < BK / UMMA_K; ++k) {
                 umma_bf16_pair(tmem_base, d0 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
                 umma_bf16_pair(tmem_base + BN, d1 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
               }
             } else {
-              for (int k = 0; k < tail; ++k) {
+              for (int k = 0; k < nk; ++k) {
                 umma_bf16_pair(tmem_base, d0 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
                 umma_bf16_pair(tmem_base + BN, d1 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
               }
             }
             chunk = (chunk + 3) % kChunks;
+            umma_commit_pair(&ctl->empty[j & 3u], 0x3);      // the stage is reusable in both CTAs once these MMAs have read it
+          }
+          if (!ok) break;
+          if (skew) {
+            if (!skewed(n_kb - skew, skew, false)) { ok = false; break; }
           } else {
+            umma_commit_pair(&ctl->acc_full[0], 0x3);
+          }
+          umma_commit_pair(&ctl->acc_full[1], 0x3);
+          ++uses0;
+          ++uses1;
+        } else {
+          const uint32_t acc_a = tmem_base + buf * BN;
+          int kb_in_seg = 0;
+          for (int kb = 0; kb < n_kb; ++kb, ++j) {
+            if (!wait_bounded(&ctl->full[j & 3u], (j >> 2) & 1u, ctl, p, WAIT_SMEM_FULL, t)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after_sync();
+            const bool full_stage = kb_in_seg != kb_seg - 1 || tail == 2 * BK / UMMA_K;
+            const uint64_t d0 = desc0 + uint64_t((((chunk + 0) % kChunks) * kChunkBytes) >> 4);
+            const uint64_t d1 = desc0 + uint64_t((((chunk + 1) % kChunks) * kChunkBytes) >> 4);
+            const uint64_t d2 = desc0 + uint64_t((((chunk + 2) % kChunks) * kChunkBytes) >> 4);
             const uint64_t d3 = desc0 + uint64_t((((chunk + 3) % kChunks) * kChunkBytes) >> 4);
+            const uint32_t first = kb != 0 ? 1u : 0u;
             if (full_stage) {
 #pragma unroll
               for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc_a, d0 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
@@ -748,17 +839,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
               }
             }
             chunk = (chunk + 4) % kChunks;
+            umma_commit_pair(&ctl->empty[j & 3u], 0x3);
+            if (++kb_in_seg == kb_seg) kb_in_seg = 0;
           }
-          umma_commit_pair(&ctl->empty[j & 3u], 0x3);      // the stage is reusable in both CTAs once these MMAs have read it
-          if (++kb_in_seg == kb_seg) kb_in_seg = 0;
-        }
-        if (!ok) break;
-        if (big) {
-          umma_commit_pair(&ctl->acc_full[0], 0x3);
-          umma_commit_pair(&ctl->acc_full[1], 0x3);
-          ++uses0;
-          ++uses1;
-        } else {
+          if (!ok) break;
           umma_commit_pair(&ctl->acc_full[buf], 0x3);
           if (buf) ++uses1; else ++uses0;
           ++small_rr;
@@ -857,6 +941,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
     tc_fence_after_sync();
     tmem_dealloc_pair(tmem_base, kTmemCols);
   }
+  clock_record.end(p);
 }
 
 // ---- host side ----------------------------------------------------------------
@@ -981,6 +1066,7 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   p.last_step = L.last_step;
   p.wait_limit_us = L.wait_limit_us ? L.wait_limit_us : (default_wait_limit_us() ? default_wait_limit_us() : 2000000u);
   p.prefetch_stages = L.prefetch_stages;
+  p.skew = L.skew < 0 ? 0 : (L.skew > 4 ? 4 : L.skew);
   p.a_hint = L.a_hint;
   p.b_hint = L.b_hint;
 

@@ -27,6 +27,9 @@ struct StatusBlock {
   int32_t detail;    // which wait gave up (WaitSite) and where
   int32_t block_idx;
   int32_t tile;
+  // written by CTA 0 of every GEMM launch that uses this block: SM cycles and nanoseconds from its start to its end
+  unsigned long long kernel_cycles;
+  unsigned long long kernel_ns;
 };
 
 enum WaitSite : int32_t {
@@ -91,6 +94,7 @@ struct GemmParams {
   uint32_t wait_limit_us;  // bound of every device-side wait
   int32_t a_hint, b_hint;  // L2 eviction priority of the A / B tile loads (ptx::L2Hint)
   int32_t prefetch_stages; // how many k-stages ahead of the shared-memory loads operands are prefetched into L2 (0 = off)
+  int32_t skew;            // 512x256 tiles: stages at each end of a tile in which accumulator 0 runs ahead of accumulator 1 (0..4)
   StatusBlock* status;
   int32_t* tile_counters;  // ring RMW only
   const uint32_t* flags;   // readiness flags (push variant), else nullptr
@@ -117,6 +121,7 @@ struct GemmLaunch {
   int a_hint = 0;   // ptx::L2Hint of the A loads
   int b_hint = 2;   // weight tiles: evict last (measured 1-2 % shorter kernels than the default priority)
   int prefetch_stages = 0;
+  int skew = 3;     // 512x256 tiles: stages at each end of a tile with accumulator 0 ahead of accumulator 1 (measured: 3 of 0..4)
   uint32_t wait_limit_us = 0;   // 0 = default bound of the device-side waits
   int last_step = 0;
   int n_blocks = 0;

@@ -123,6 +123,16 @@ def test_selector_hand_example_and_errors():
     assert lib.compass_select(C.byref(bad), C.byref(cal), C.byref(out)) == api.ERR_SHAPE
 
 
+def test_read_kernel_clock_rejects_null_arguments_before_touching_a_device():
+    lib = api.lib()
+    cycles, ns = C.c_uint64(7), C.c_uint64(7)
+    assert lib.compass_read_kernel_clock(None, None, C.byref(cycles), C.byref(ns)) == api.ERR_INVALID_ARG
+    fake_ws = C.c_void_p(4096)                       # never dereferenced: the NULL checks come first
+    assert lib.compass_read_kernel_clock(fake_ws, None, None, C.byref(ns)) == api.ERR_INVALID_ARG
+    assert lib.compass_read_kernel_clock(fake_ws, None, C.byref(cycles), None) == api.ERR_INVALID_ARG
+    assert (cycles.value, ns.value) == (7, 7)
+
+
 def test_calibration_matches_oracle():
     alpha, beta = 1.07, 0.025
     tc, tm, d, t = [], [], [], []

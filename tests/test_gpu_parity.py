@@ -42,6 +42,22 @@ def test_library_was_loaded_and_counts_launches():
     check_all(outs, ops.ag_gemm(A, B), w.name)
 
 
+def test_kernel_clock_record_is_plausible():
+    """CTA 0 records its cycles and nanoseconds: their ratio must be an SM clock a B200 can have."""
+    w = small(wl.OP_AG_GEMM, 4, 512, 1024, 2048)
+    A_bits, B_bits = wl.make_inputs(w)
+    pr = api.make_problem(w.op, w.P, w.M, w.N, w.K)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    ws = api.alloc_workspace(pr)
+    assert api.compass_read_kernel_clock(ws) == (0, 0)
+    api.compass_ag_gemm(pr, A, B, [o.view for o in outs], ws)
+    cycles, ns = api.compass_read_kernel_clock(ws)
+    assert cycles > 0 and ns > 0
+    assert 300.0 < cycles / ns * 1e3 < 2500.0          # MHz
+    assert api.compass_read_status(ws) == (api.OK, 0)
+
+
 def test_config1_ag_gemm_full():
     w = wl.C1_AG
     A, B = wl.make_inputs(w)
@@ -92,6 +108,13 @@ def test_gemm_rs_small_shapes(P, m, N, K, rings):
     (wl.OP_AG_GEMM, 4, 1024, 2568, 72, api.ORDER_STEP_MAJOR),
     (wl.OP_GEMM_RS, 8, 1024, 2568, 88, api.ORDER_RANK_MAJOR),
     (wl.OP_AG_GEMM, 2, 1536, 5128, 64, api.ORDER_RANK_MAJOR),      # 768-row partitions: 512-row tiles do not divide them
+    # k-stage counts around the point where the two accumulators of a 512x256 tile start to be
+    # issued skewed at the tile's ends (5, 6 and 7 stages, the last one partial; then a long loop)
+    (wl.OP_AG_GEMM, 4, 1024, 2568, 320, api.ORDER_RANK_MAJOR),
+    (wl.OP_AG_GEMM, 4, 1024, 2568, 384, api.ORDER_RANK_MAJOR),
+    (wl.OP_AG_GEMM, 4, 1024, 2568, 424, api.ORDER_STEP_MAJOR),
+    (wl.OP_AG_GEMM, 4, 1024, 2568, 1032, api.ORDER_RANK_MAJOR),
+    (wl.OP_GEMM_RS, 4, 1024, 2568, 104, api.ORDER_RANK_MAJOR),     # 4 segments x 2 stages, every segment with a partial stage
 ])
 def test_big_and_small_tiles_in_one_launch(op, P, m, N, K, order):
     w = small(op, P, m, N, K, dist=0.05)
