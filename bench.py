@@ -530,6 +530,7 @@ def run_ours(args, w_ag, w_rs):
                          "frac": achieved / peak, "traffic": traffic,
                          "peak_source": f"{'sustained' if sustained else 'burst'} cuBLAS bf16, of {peak_src}",
                          "kernel": "gemm_mixed_kernel (two launches per step: AG-GEMM and GEMM-RS)",
+                         "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
                          "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS},
             "ag_gemm": {"ms": t_ag, "ms_median": float(np.median(ag_ms)), "ms_best": float(np.min(ag_ms)),
                         "tflops": w_ag.flops / (t_ag * 1e-3) / 1e12,

@@ -40,8 +40,20 @@ __global__ void __launch_bounds__(256) reduce_partials_kernel(const __grid_const
     const int64_t col = w - row * p.n_vec;
     const int64_t src = (int64_t(c) * p.m + p.slice_begin + row) * p.n_vec + col;
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    // four ranks' vectors are fetched before the first is added, so that a thread keeps 64 bytes in flight
+    int q = 0;
+    for (; q + 4 <= p.P; q += 4) {
+      const uint4 v0 = __ldg(p.partial[q] + src);
+      const uint4 v1 = __ldg(p.partial[q + 1] + src);
+      const uint4 v2 = __ldg(p.partial[q + 2] + src);
+      const uint4 v3 = __ldg(p.partial[q + 3] + src);
+      accumulate_bf16x8(acc, v0);
+      accumulate_bf16x8(acc, v1);
+      accumulate_bf16x8(acc, v2);
+      accumulate_bf16x8(acc, v3);
+    }
 #pragma unroll 1
-    for (int q = 0; q < p.P; ++q) {
+    for (; q < p.P; ++q) {
       const uint4 v = __ldg(p.partial[q] + src);
       accumulate_bf16x8(acc, v);
     }
