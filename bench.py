@@ -212,6 +212,39 @@ def workload_config(w_ag, w_rs):
 # ---------------------------------------------------------------------------------
 # InterDecom sweep, calibration of the models, strategy selection (reported beside the headline number)
 
+def mlp_report(torch, api):
+    """The chained MLP block (Section II-A: AllGather -> GEMM0 -> GEMM1 -> ReduceScatter) on the 7B shape:
+    two fused kernels back to back through compass_mlp_block, SwiGLU applied in the first kernel's epilogue."""
+    w = wl.MLP_7B
+    stream = torch.cuda.current_stream()
+    X, W0, W1 = wl.make_mlp_inputs(w)
+    dX, dW0, dW1 = [api.to_device(a) for a in X], [api.to_device(a) for a in W0], [api.to_device(a) for a in W1]
+    H = [torch.empty((w.M, w.hc), dtype=torch.bfloat16, device="cuda") for _ in range(w.P)]
+    out = [torch.empty((w.m, w.hidden), dtype=torch.bfloat16, device="cuda") for _ in range(w.P)]
+    mp = api.make_mlp(w.P, w.M, w.hidden, w.ffn, activation=w.activation)
+    ws = api.alloc_mlp_workspace(mp)
+    run = lambda: api.compass_mlp_block(mp, dX, dW0, H, dW1, out, ws, stream)
+    for _ in range(5):
+        run()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(30):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        run()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    status = api.compass_read_status(ws)
+    if status != (api.OK, 0):
+        raise SystemExit(f"device-side status after the MLP block: {status}")
+    med = float(np.median(ts))
+    return {"workload": f"{w.name} (P={w.P}, M={w.M}, hidden={w.hidden}, ffn={w.ffn}/rank interleaved gate/up)",
+            "ms_median": med, "ms_best": float(np.min(ts)), "tflops": w.flops / (med * 1e-3) / 1e12,
+            "frac_of_nominal_2250": w.flops / (med * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS,
+            "kernels_per_call": 2, "intermediate_bytes": 2 * w.P * w.M * w.hc}
+
+
 def interdecom_report(torch, api, hbm_gbs):
     """Times compass_decomp for d in {1,2,4,8,16} on the config-4 shapes, fits
     the models' parameters on other shapes (Section IV-C: one-time offline
@@ -547,6 +580,8 @@ def run_ours(args, w_ag, w_rs):
         }
         if world == 1 and not args.no_sweep:
             del hag, hrs
+            torch.cuda.empty_cache()
+            line["mlp_block"] = mlp_report(torch, api)
             torch.cuda.empty_cache()
             line["interdecom"] = interdecom_report(torch, api, peaks["hbm_gbs"])
         if world == 1 and not args.no_cpu_baseline:

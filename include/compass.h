@@ -225,6 +225,47 @@ int compass_decomp(const compass_problem* problem, const void* const* A, const v
  * Host arithmetic only. */
 int compass_select(const compass_problem* problem, const compass_calib* calib, compass_choice* out);
 
+/* ---- the tensor-parallel MLP block (Section II-A, the two-layer MLP figure) --
+ * AllGather -> GEMM0 (W0 column-parallel) -> GEMM1 (W1 row-parallel) ->
+ * ReduceScatter as TWO fused kernels back to back on one stream: the fused
+ * AllGather+GEMM with the element-wise function applied to the FP32
+ * accumulator in its epilogue, then the fused GEMM+ReduceScatter reading the
+ * BF16 result:
+ *     H_r   = act( gather(X) * W0_r )
+ *     Out_c = rows [c*M/P, (c+1)*M/P) of  sum_q H_q * W1_q
+ * The paper's text puts nothing between the two GEMMs (COMPASS_ACT_NONE); an
+ * MLP has an activation there, so two are offered:
+ *   GELU_TANH: 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))
+ *   SWIGLU:    the rows of W0_r alternate (gate_0, up_0, gate_1, up_1, ...), so
+ *              that GEMM0's columns 2j and 2j+1 are gate_j and up_j;
+ *              H[:, j] = gate_j / (1 + exp(-gate_j)) * up_j and H has ffn / 2
+ *              columns (ffn must be a multiple of 16).
+ *   X:   P device pointers, X[r]  = [M/P x hidden]
+ *   W0:  P device pointers, W0[r] = [ffn x hidden]       (K-major, as every weight)
+ *   H:   P device pointers, H[r]  = [M x hc], hc = ffn (ffn / 2 with SWIGLU);
+ *        caller-owned intermediate, every element is written
+ *   W1:  P device pointers, W1[r] = [hidden x hc]
+ *   Out: P device pointers, Out[r] = [M/P x hidden]
+ *   workspace: >= compass_mlp_workspace_bytes bytes, 256-byte aligned, zeroed
+ *   once with compass_workspace_init; compass_read_status reports a bounded
+ *   wait of either kernel that gave up. */
+enum { COMPASS_ACT_NONE = 0, COMPASS_ACT_GELU_TANH = 1, COMPASS_ACT_SWIGLU = 2 };
+typedef struct compass_mlp {
+  int32_t P;           /* tensor-parallel size */
+  int32_t rings;       /* 1 or 2, as in compass_problem */
+  int64_t M;           /* rows of the gathered input (all ranks) */
+  int64_t hidden;      /* K of GEMM0 = N of GEMM1 */
+  int64_t ffn;         /* N of GEMM0 per rank */
+  int32_t activation;  /* COMPASS_ACT_* */
+  int32_t rs_variant;  /* COMPASS_RS_* of the second kernel */
+  int32_t order;       /* COMPASS_ORDER_* of the first kernel */
+  int32_t reserved;    /* 0 */
+} compass_mlp;
+int compass_mlp_workspace_bytes(const compass_mlp* mlp, size_t* bytes);
+int compass_mlp_block(const compass_mlp* mlp, const void* const* X, const void* const* W0, void* const* H,
+                      const void* const* W1, void* const* Out, void* workspace, size_t workspace_bytes,
+                      void* cuda_stream);
+
 /* ---- models, individually (host) ----------------------------------------- */
 /* Eq. 2-3: (d-1)*max(T_comp,T_comm)/d*(alpha+beta*d) + T_comp/d + T_comm/d. */
 int compass_model_decomp_time(double t_comp, double t_comm, double alpha, double beta, int d, double* out);

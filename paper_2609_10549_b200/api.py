@@ -25,6 +25,7 @@ STRATEGY_INTRAFUSION, STRATEGY_INTERDECOM = 0, 1
 ORDER_RANK_MAJOR, ORDER_STEP_MAJOR = 0, 1
 COPY_KERNEL, COPY_ENGINES = 0, 1
 WS_FUSED, WS_DECOMP, WS_PUSH = 0, 1, 2
+ACT_NONE, ACT_GELU_TANH, ACT_SWIGLU = 0, 1, 2
 MAX_P = 16
 STATUS_BYTES = 256
 
@@ -36,6 +37,7 @@ EXPORTS = (
     "compass_read_status", "compass_launch_plan", "compass_fused_host", "compass_status_string",
     "compass_last_cuda_error", "compass_kernel_launch_count", "compass_gemm_rs_sequential_noalloc",
     "compass_set_wait_limit_us", "compass_calib_fit_line", "compass_ag_gemm_push", "compass_read_kernel_clock",
+    "compass_mlp_workspace_bytes", "compass_mlp_block",
 )
 
 
@@ -49,6 +51,11 @@ class Problem(C.Structure):
     _fields_ = [("op", C.c_int32), ("P", C.c_int32), ("rings", C.c_int32), ("d", C.c_int32),
                 ("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64),
                 ("dtype", C.c_int32), ("rs_variant", C.c_int32), ("order", C.c_int32), ("copy_mode", C.c_int32)]
+
+
+class Mlp(C.Structure):
+    _fields_ = [("P", C.c_int32), ("rings", C.c_int32), ("M", C.c_int64), ("hidden", C.c_int64), ("ffn", C.c_int64),
+                ("activation", C.c_int32), ("rs_variant", C.c_int32), ("order", C.c_int32), ("reserved", C.c_int32)]
 
 
 class SchedEntry(C.Structure):
@@ -87,6 +94,8 @@ def lib() -> C.CDLL:
             getattr(L, name).argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p]
         L.compass_decomp.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.compass_ag_gemm_push.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.compass_mlp_workspace_bytes.argtypes = [C.POINTER(Mlp), C.POINTER(C.c_size_t)]
+        L.compass_mlp_block.argtypes = [C.POINTER(Mlp), pp, pp, pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p]
         L.compass_select.argtypes = [C.POINTER(Problem), C.POINTER(Calib), C.POINTER(Choice)]
         L.compass_model_decomp_time.argtypes = [C.c_double] * 4 + [C.c_int, C.POINTER(C.c_double)]
         L.compass_model_optimal_degree.argtypes = [C.c_double] * 4 + [C.c_int, C.c_int, C.POINTER(C.c_int),
@@ -279,6 +288,32 @@ def compass_ag_gemm_push(problem: Problem, A: Sequence, B: Sequence, Cout: Seque
     p, n = _ws(workspace)
     _check(lib().compass_ag_gemm_push(C.byref(problem), _ptr_array(A), _ptr_array(B), _ptr_array(Cout), p, n,
                                       _stream_handle(stream_compute), _stream_handle(stream_copy)), "compass_ag_gemm_push")
+
+
+def make_mlp(P: int, M: int, hidden: int, ffn: int, activation: int = 0, rings: int = 2,
+             rs_variant: int = RS_SEGMENTED_K, order: int = ORDER_RANK_MAJOR) -> Mlp:
+    return Mlp(P=P, rings=rings, M=M, hidden=hidden, ffn=ffn, activation=activation, rs_variant=rs_variant,
+               order=order, reserved=0)
+
+
+def compass_mlp_workspace_bytes(mlp: Mlp) -> int:
+    n = C.c_size_t(0)
+    _check(lib().compass_mlp_workspace_bytes(C.byref(mlp), C.byref(n)), "compass_mlp_workspace_bytes")
+    return int(n.value)
+
+
+def alloc_mlp_workspace(mlp: Mlp, device="cuda"):
+    import torch
+    ws = torch.empty(compass_mlp_workspace_bytes(mlp), dtype=torch.uint8, device=device)
+    compass_workspace_init(ws)
+    return ws
+
+
+def compass_mlp_block(mlp: Mlp, X: Sequence, W0: Sequence, H: Sequence, W1: Sequence, Out: Sequence, workspace,
+                      stream=None) -> None:
+    p, n = _ws(workspace)
+    _check(lib().compass_mlp_block(C.byref(mlp), _ptr_array(X), _ptr_array(W0), _ptr_array(H), _ptr_array(W1),
+                                   _ptr_array(Out), p, n, _stream_handle(stream)), "compass_mlp_block")
 
 
 def compass_decomp(problem: Problem, A: Sequence, B: Sequence, out: Sequence, workspace, stream_compute=None,

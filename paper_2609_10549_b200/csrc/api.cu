@@ -235,6 +235,40 @@ int fused_call(const compass_problem* pr, int op, const void* const* A, const vo
   return launch_gemm(L, static_cast<cudaStream_t>(stream));
 }
 
+// ---- MLP block -----------------------------------------------------------------
+
+// The two fused operators of the block as problems of their own.
+int mlp_problems(const compass_mlp* mp, compass_problem* ag, compass_problem* rs) {
+  if (mp == nullptr) return COMPASS_ERR_INVALID_ARG;
+  if (mp->activation != COMPASS_ACT_NONE && mp->activation != COMPASS_ACT_GELU_TANH && mp->activation != COMPASS_ACT_SWIGLU)
+    return COMPASS_ERR_INVALID_ARG;
+  if (mp->reserved != 0) return COMPASS_ERR_INVALID_ARG;
+  if (mp->hidden <= 0 || mp->ffn <= 0) return COMPASS_ERR_SHAPE;
+  // SwiGLU: (gate, up) column pairs; the result's rows must still be a multiple of 16 bytes for the second GEMM's loads
+  if (mp->activation == COMPASS_ACT_SWIGLU && mp->ffn % 16 != 0) return COMPASS_ERR_ALIGNMENT;
+  std::memset(ag, 0, sizeof(*ag));
+  ag->op = COMPASS_OP_AG_GEMM;
+  ag->P = mp->P;
+  ag->rings = mp->rings;
+  ag->d = 1;
+  ag->M = mp->M;
+  ag->N = mp->ffn;
+  ag->K = mp->hidden;
+  ag->dtype = COMPASS_DTYPE_BF16;
+  ag->rs_variant = COMPASS_RS_SEGMENTED_K;
+  ag->order = mp->order;
+  ag->copy_mode = COMPASS_COPY_KERNEL;
+  *rs = *ag;
+  rs->op = COMPASS_OP_GEMM_RS;
+  rs->N = mp->hidden;
+  rs->K = mp->activation == COMPASS_ACT_SWIGLU ? mp->ffn / 2 : mp->ffn;
+  rs->rs_variant = mp->rs_variant;
+  int st = validate_problem(ag, COMPASS_OP_AG_GEMM, false);
+  if (st != COMPASS_OK) return st;
+  return validate_problem(rs, COMPASS_OP_GEMM_RS, false);
+}
+
+
 // ---- InterDecom ----------------------------------------------------------------
 
 // Events that order the two streams of a call; created on first use, one set per device
@@ -484,6 +518,65 @@ static StreamWriteValue32Fn stream_write_fn() {
       fn = reinterpret_cast<StreamWriteValue32Fn>(ptr);
   }
   return fn;
+}
+
+extern "C" int compass_mlp_workspace_bytes(const compass_mlp* mp, size_t* bytes) {
+  if (bytes == nullptr) return COMPASS_ERR_INVALID_ARG;
+  compass_problem ag, rs;
+  int st = mlp_problems(mp, &ag, &rs);
+  if (st != COMPASS_OK) return st;
+  size_t a = 0, b = 0;
+  st = compass_workspace_bytes(&ag, COMPASS_WS_FUSED, &a);
+  if (st != COMPASS_OK) return st;
+  st = compass_workspace_bytes(&rs, COMPASS_WS_FUSED, &b);
+  if (st != COMPASS_OK) return st;
+  *bytes = a > b ? a : b;      // the two launches are ordered on one stream and share status block and counters
+  return COMPASS_OK;
+}
+
+extern "C" int compass_mlp_block(const compass_mlp* mp, const void* const* X, const void* const* W0, void* const* H,
+                                 const void* const* W1, void* const* Out, void* ws, size_t ws_bytes, void* stream) {
+  compass_problem ag, rs;
+  int st = mlp_problems(mp, &ag, &rs);
+  if (st != COMPASS_OK) return st;
+  st = validate_pointers(X, W0, H, mp->P);
+  if (st != COMPASS_OK) return st;
+  st = validate_pointers(H, W1, Out, mp->P);
+  if (st != COMPASS_OK) return st;
+  size_t need = 0;
+  st = compass_mlp_workspace_bytes(mp, &need);
+  if (st != COMPASS_OK) return st;
+  if (ws == nullptr) return COMPASS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0) return COMPASS_ERR_ALIGNMENT;
+  if (ws_bytes < need) return COMPASS_ERR_BUFFER_TOO_SMALL;
+
+  static thread_local GemmLaunch L;
+  // AllGather + GEMM0, the activation applied in the epilogue: H_r = act(gather(X) * W0_r)
+  st = plan_fused(&ag, &L, nullptr);
+  if (st != COMPASS_OK) return st;
+  for (int r = 0; r < mp->P; ++r) {
+    L.a_ptr[r] = X[r];
+    L.b_ptr[r] = W0[r];
+    L.out_ptr[r] = H[r];
+  }
+  L.activation = mp->activation;
+  L.ldo = rs.K;                                  // H's row pitch: ffn, or ffn / 2 with SwiGLU
+  L.status = static_cast<StatusBlock*>(ws);
+  L.tile_counters = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + COMPASS_STATUS_BYTES);
+  st = launch_gemm(L, static_cast<cudaStream_t>(stream));
+  L.activation = ACT_NONE;                       // the launch descriptor is reused by the next call on this thread
+  if (st != COMPASS_OK) return st;
+  // GEMM1 + ReduceScatter on the stream-ordered result
+  st = plan_fused(&rs, &L, nullptr);
+  if (st != COMPASS_OK) return st;
+  for (int r = 0; r < mp->P; ++r) {
+    L.a_ptr[r] = H[r];
+    L.b_ptr[r] = W1[r];
+    L.out_ptr[r] = Out[r];
+  }
+  L.status = static_cast<StatusBlock*>(ws);
+  L.tile_counters = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + COMPASS_STATUS_BYTES);
+  return launch_gemm(L, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int compass_ag_gemm_push(const compass_problem* pr, const void* const* A, const void* const* B, void* const* C,

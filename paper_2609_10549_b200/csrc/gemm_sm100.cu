@@ -90,6 +90,17 @@ __device__ __forceinline__ void report_timeout(const GemmParams& p, Control* ctl
   }
 }
 
+// Activations of the MLP block's first GEMM, on the FP32 accumulator.  exp through the fast
+// exponential (relative error ~2^-21, far below the BF16 rounding that follows).
+__device__ __forceinline__ float gelu_tanh_f32(float x) {
+  const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+  const float t = 1.0f - __fdividef(2.0f, 1.0f + __expf(2.0f * u));       // tanh(u); exp overflow gives exactly 1
+  return 0.5f * x * (1.0f + t);
+}
+__device__ __forceinline__ float swiglu_f32(float gate, float up) {
+  return __fdividef(gate, 1.0f + __expf(-gate)) * up;                     // silu(gate) * up
+}
+
 // CTA 0 records how many SM cycles and nanoseconds it ran: their ratio is the clock the
 // kernel really had (under a power cap well below the nominal one).
 struct ClockRecord {
@@ -211,7 +222,8 @@ struct StageIter {
   }
 };
 
-template <bool kPair>
+// kAct: the plain-store epilogue applies p.activation (its own instantiation, see gemm_mixed_kernel).
+template <bool kPair, bool kAct>
 __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
   using C = Cfg<kPair>;
   extern __shared__ uint8_t smem_raw[];
@@ -425,7 +437,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       const bool row_ok = row_in_block < p.rows_per_block;
       const int ncols = min(BN, p.N - tc.nt * BN);
       const int nchunks = (ncols + 31) >> 5;
-      __nv_bfloat16* orow = p.out[b.out_idx] + int64_t(b.out_row0 + row_in_block) * p.ldo + int64_t(tc.nt) * BN;
+      // SwiGLU halves the columns: accumulator columns (2j, 2j+1) = (gate, up) give output column j
+      const int act = kAct ? p.activation : int(ACT_NONE);
+      const int oshift = act == ACT_SWIGLU ? 1 : 0;
+      __nv_bfloat16* orow = p.out[b.out_idx] + int64_t(b.out_row0 + row_in_block) * p.ldo + ((int64_t(tc.nt) * BN) >> oshift);
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
 
       // Ring read-modify-write: contributor `step` of a partition adds its
@@ -485,12 +500,23 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                   f[6] += __uint_as_float(o.w << 16);
                   f[7] += __uint_as_float(o.w & 0xFFFF0000u);
                 }
-                uint4 q;
-                q.x = pack_bf16x2(f[0], f[1]);
-                q.y = pack_bf16x2(f[2], f[3]);
-                q.z = pack_bf16x2(f[4], f[5]);
-                q.w = pack_bf16x2(f[6], f[7]);
-                *reinterpret_cast<uint4*>(orow + c * 32 + g * 8) = q;
+                if (act == ACT_SWIGLU) {
+                  uint2 h;
+                  h.x = pack_bf16x2(swiglu_f32(f[0], f[1]), swiglu_f32(f[2], f[3]));
+                  h.y = pack_bf16x2(swiglu_f32(f[4], f[5]), swiglu_f32(f[6], f[7]));
+                  *reinterpret_cast<uint2*>(orow + ((c * 32 + g * 8) >> 1)) = h;
+                } else {
+                  if (act == ACT_GELU_TANH) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) f[i] = gelu_tanh_f32(f[i]);
+                  }
+                  uint4 q;
+                  q.x = pack_bf16x2(f[0], f[1]);
+                  q.y = pack_bf16x2(f[2], f[3]);
+                  q.z = pack_bf16x2(f[4], f[5]);
+                  q.w = pack_bf16x2(f[6], f[7]);
+                  *reinterpret_cast<uint4*>(orow + c * 32 + g * 8) = q;
+                }
               }
             }
           }
@@ -617,6 +643,9 @@ struct MixedIter {
   }
 };
 
+// kAct: the epilogue applies p.activation.  A separate instantiation, because the extra code in the
+// accumulator-read phase (which the MMA issuer waits for) slows the plain store down by 1-3 %.
+template <bool kAct>
 __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -879,7 +908,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
         // big: this CTA owns rows [256*rank, +256) of the tile, accumulator a holds its 128-row block a
         const int row_in_block = tile.row0 + (tile.big ? int(cta_rank) * 2 * BM + a * BM : int(cta_rank) * BM) + quarter * 32 + lane;
         const bool row_ok = row_in_block < p.rows_per_block;
-        __nv_bfloat16* orow = p.out[b.out_idx] + int64_t(b.out_row0 + row_in_block) * p.ldo + int64_t(tile.nt) * BN;
+        // SwiGLU halves the columns: accumulator columns (2j, 2j+1) = (gate, up) give output column j
+        const int act = kAct ? p.activation : int(ACT_NONE);
+        const int oshift = act == ACT_SWIGLU ? 1 : 0;
+        const int ocols = ncols >> oshift;
+        __nv_bfloat16* orow = p.out[b.out_idx] + int64_t(b.out_row0 + row_in_block) * p.ldo + ((int64_t(tile.nt) * BN) >> oshift);
         const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
         const int first_row = row_in_block - lane;          // row of lane 0
         __nv_bfloat16* obase = orow - int64_t(lane) * p.ldo;
@@ -893,10 +926,28 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
           tmem_ld_32x32b_x32(taddr + c * 64, v);
           tmem_ld_32x32b_x32(taddr + c * 64 + 32, w);
           tmem_ld_wait();
+          if (act == ACT_SWIGLU) {
+            // 64 accumulator columns -> 32 output columns, packed densely from register 0 on
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            packed[c * 32 + i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-            packed[c * 32 + 16 + i] = pack_bf16x2(__uint_as_float(w[2 * i]), __uint_as_float(w[2 * i + 1]));
+            for (int i = 0; i < 8; ++i) {
+              packed[c * 16 + i] = pack_bf16x2(swiglu_f32(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1])),
+                                               swiglu_f32(__uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3])));
+              packed[c * 16 + 8 + i] = pack_bf16x2(swiglu_f32(__uint_as_float(w[4 * i]), __uint_as_float(w[4 * i + 1])),
+                                                   swiglu_f32(__uint_as_float(w[4 * i + 2]), __uint_as_float(w[4 * i + 3])));
+            }
+          } else {
+            if (act == ACT_GELU_TANH) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                v[i] = __float_as_uint(gelu_tanh_f32(__uint_as_float(v[i])));
+                w[i] = __float_as_uint(gelu_tanh_f32(__uint_as_float(w[i])));
+              }
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              packed[c * 32 + i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+              packed[c * 32 + 16 + i] = pack_bf16x2(__uint_as_float(w[2 * i]), __uint_as_float(w[2 * i + 1]));
+            }
           }
         }
         tc_fence_before_sync();
@@ -904,7 +955,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
         if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->acc_empty[buf]), 0));
         // 2) registers -> padded shared memory -> global, 64 columns per pass: every store
         //    instruction writes 4 rows x 128 contiguous bytes.
-        const int npass = (ncols + 63) >> 6;
+        const int npass = (ocols + 63) >> 6;
         const int seg = lane & 7;
 #pragma unroll
         for (int pass = 0; pass < BN / 64; ++pass) {
@@ -919,7 +970,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               const int r = i * 4 + (lane >> 3);
-              if (first_row + r < p.rows_per_block && col < ncols) {
+              if (first_row + r < p.rows_per_block && col < ocols) {
                 const uint4 q = *reinterpret_cast<const uint4*>(stage + r * kStageRowBytes + seg * 16);
                 *reinterpret_cast<uint4*>(obase + int64_t(r) * p.ldo + col) = q;
               }
@@ -1000,11 +1051,17 @@ int device_info(DeviceInfo** out) {
   if (!info.ready) {
     e = cudaDeviceGetAttribute(&info.num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return record_cuda_error(e);
-    e = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<false>()));
+    e = cudaFuncSetAttribute(gemm_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<false>()));
     if (e != cudaSuccess) return record_cuda_error(e);
-    e = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<true>()));
+    e = cudaFuncSetAttribute(gemm_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<false>()));
     if (e != cudaSuccess) return record_cuda_error(e);
-    e = cudaFuncSetAttribute(gemm_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kMixedSmemBytes));
+    e = cudaFuncSetAttribute(gemm_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<true>()));
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaFuncSetAttribute(gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<true>()));
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaFuncSetAttribute(gemm_mixed_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kMixedSmemBytes));
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaFuncSetAttribute(gemm_mixed_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kMixedSmemBytes));
     if (e != cudaSuccess) return record_cuda_error(e);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(unsigned(info.num_sms / 2 * 2));
@@ -1018,7 +1075,7 @@ int device_info(DeviceInfo** out) {
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int clusters = 0;
-    e = cudaOccupancyMaxActiveClusters(&clusters, gemm_kernel<true>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&clusters, gemm_kernel<true, false>, &cfg);
     if (e != cudaSuccess) return record_cuda_error(e);
     info.max_pairs = clusters;
     info.ready = true;
@@ -1041,6 +1098,9 @@ int gemm_tile_rows(int mode, int rows_per_block) {
 
 int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   static thread_local GemmParams p;
+  // an activation goes with the plain store only (the ring read-modify-write adds partial sums)
+  if (L.activation != ACT_NONE && L.epilogue != EPI_STORE) return COMPASS_ERR_INVALID_ARG;
+  if (L.activation == ACT_SWIGLU && (L.N % 16 != 0 || L.ldo < L.N / 2)) return COMPASS_ERR_INVALID_ARG;
   const int tile_rows = gemm_tile_rows(L.mode, L.rows_per_block);
   const bool pair = tile_rows == 2 * BM;
   const int b_box_rows = pair ? BN / 2 : BN;
@@ -1066,6 +1126,7 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   p.last_step = L.last_step;
   p.wait_limit_us = L.wait_limit_us ? L.wait_limit_us : (default_wait_limit_us() ? default_wait_limit_us() : 2000000u);
   p.prefetch_stages = L.prefetch_stages;
+  p.activation = L.activation;
   p.skew = L.skew < 0 ? 0 : (L.skew > 4 ? 4 : L.skew);
   p.a_hint = L.a_hint;
   p.b_hint = L.b_hint;
@@ -1109,7 +1170,10 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    e = mixed ? cudaLaunchKernelEx(&cfg, gemm_mixed_kernel, p) : cudaLaunchKernelEx(&cfg, gemm_kernel<true>, p);
+    if (mixed && L.activation != ACT_NONE) e = cudaLaunchKernelEx(&cfg, gemm_mixed_kernel<true>, p);
+    else if (mixed) e = cudaLaunchKernelEx(&cfg, gemm_mixed_kernel<false>, p);
+    else if (L.activation != ACT_NONE) e = cudaLaunchKernelEx(&cfg, gemm_kernel<true, true>, p);
+    else e = cudaLaunchKernelEx(&cfg, gemm_kernel<true, false>, p);
   } else {
     if (pair) {   // no room for clusters on this device: fall back to single-CTA tiles
       p.tiles_m = (L.rows_per_block + BM - 1) / BM;
@@ -1120,7 +1184,8 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
         if (!encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, BN)) return record_cuda_error(cudaErrorUnknown);
     }
     const int grid = p.total_tiles < info->num_sms ? p.total_tiles : info->num_sms;
-    gemm_kernel<false><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);
+    if (L.activation != ACT_NONE) gemm_kernel<false, true><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);
+    else gemm_kernel<false, false><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);
     e = cudaGetLastError();
   }
   count_kernel_launch();

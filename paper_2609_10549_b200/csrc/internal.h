@@ -32,6 +32,9 @@ struct StatusBlock {
   unsigned long long kernel_ns;
 };
 
+// Element-wise function between the accumulator and the store (values of COMPASS_ACT_*).
+enum ActivationMode : int32_t { ACT_NONE = 0, ACT_GELU_TANH = 1, ACT_SWIGLU = 2 };
+
 enum WaitSite : int32_t {
   WAIT_NONE = 0,
   WAIT_SMEM_EMPTY = 1,     // TMA producer waiting for a free pipeline stage
@@ -94,6 +97,7 @@ struct GemmParams {
   uint32_t wait_limit_us;  // bound of every device-side wait
   int32_t a_hint, b_hint;  // L2 eviction priority of the A / B tile loads (ptx::L2Hint)
   int32_t prefetch_stages; // how many k-stages ahead of the shared-memory loads operands are prefetched into L2 (0 = off)
+  int32_t activation;      // ActivationMode applied to the FP32 accumulator before the BF16 store (plain-store epilogue only)
   int32_t skew;            // 512x256 tiles: stages at each end of a tile in which accumulator 0 runs ahead of accumulator 1 (0..4)
   StatusBlock* status;
   int32_t* tile_counters;  // ring RMW only
@@ -121,6 +125,7 @@ struct GemmLaunch {
   int a_hint = 0;   // ptx::L2Hint of the A loads
   int b_hint = 2;   // weight tiles: evict last (measured 1-2 % shorter kernels than the default priority)
   int prefetch_stages = 0;
+  int activation = 0;   // ActivationMode
   int skew = 3;     // 512x256 tiles: stages at each end of a tile with accumulator 0 ahead of accumulator 1 (measured: 3 of 0..4)
   uint32_t wait_limit_us = 0;   // 0 = default bound of the device-side waits
   int last_step = 0;

@@ -146,3 +146,50 @@ def make_structured_inputs(w: Workload, kind: str) -> Tuple[List[np.ndarray], Li
         A.append(f32_to_bf16_bits(a))
         B.append(f32_to_bf16_bits(b))
     return A, B
+
+
+# ---- the tensor-parallel MLP block (Section II-A) ---------------------------------
+
+ACT_NONE, ACT_GELU_TANH, ACT_SWIGLU = 0, 1, 2
+
+
+@dataclass(frozen=True)
+class MlpWorkload:
+    """X_r [M/P x hidden], W0_r [ffn x hidden] (column-parallel slice, K-major), W1_r [hidden x hc]
+    (row-parallel slice, K-major); hc = ffn, or ffn / 2 when the activation pairs (gate, up) columns."""
+    name: str
+    P: int
+    M: int
+    hidden: int
+    ffn: int                 # GEMM0 output columns per rank
+    activation: int = ACT_NONE
+    seed: int = 0
+
+    @property
+    def m(self) -> int:
+        return self.M // self.P
+
+    @property
+    def hc(self) -> int:
+        return self.ffn // 2 if self.activation == ACT_SWIGLU else self.ffn
+
+    @property
+    def flops(self) -> float:
+        """FLOPs of both GEMMs over all P logical ranks."""
+        return 2.0 * self.P * self.M * self.hidden * (self.ffn + self.hc)
+
+
+def make_mlp_inputs(w: MlpWorkload) -> Tuple[List[np.ndarray], List[np.ndarray], List[np.ndarray]]:
+    """(X, W0, W1) as BF16 bit patterns.  X ~ N(0, 1); the weights' standard deviations keep both GEMMs'
+    outputs of order one: 1/sqrt(hidden) for W0, 1/sqrt(P * hc) for W1."""
+    s0 = 1.0 / float(np.sqrt(w.hidden))
+    s1 = 1.0 / float(np.sqrt(w.P * w.hc))
+    X = [_draw((w.m, w.hidden), ("normal", 1.0), tensor_seed(w.seed, r, 0)) for r in range(w.P)]
+    W0 = [_draw((w.ffn, w.hidden), ("normal", s0), tensor_seed(w.seed, r, 1)) for r in range(w.P)]
+    W1 = [_draw((w.hidden, w.hc), ("normal", s1), tensor_seed(w.seed, r, 2)) for r in range(w.P)]
+    return X, W0, W1
+
+
+# LLaMA-7B MLP over 8 ranks: hidden 4096, 11008 / 8 = 1376 gate and up columns per rank (interleaved rows of
+# W0_r), 8192 tokens.  Its second GEMM is the GEMM+ReduceScatter of configuration 3.
+MLP_7B = MlpWorkload("MLP-7B-SwiGLU", P=8, M=8192, hidden=4096, ffn=2752, activation=ACT_SWIGLU)

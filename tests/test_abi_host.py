@@ -35,6 +35,8 @@ def test_struct_layouts_match_the_header():
     assert C.sizeof(api.Calib) == 64
     assert C.sizeof(api.Choice) == 8 + 6 * 8
     assert C.sizeof(api.PlanBlock) == 44
+    assert C.sizeof(api.Mlp) == 2 * 4 + 3 * 8 + 4 * 4
+    assert api.Mlp.M.offset == 8 and api.Mlp.activation.offset == 32
 
 
 @pytest.mark.parametrize("op", [OP_AG_GEMM, OP_GEMM_RS])
@@ -121,6 +123,42 @@ def test_selector_hand_example_and_errors():
     assert lib.compass_select(C.byref(pr), None, C.byref(out)) == api.ERR_INVALID_ARG
     bad = api.make_problem(OP_AG_GEMM, 3, 4096, N, K)
     assert lib.compass_select(C.byref(bad), C.byref(cal), C.byref(out)) == api.ERR_SHAPE
+
+
+def test_mlp_block_argument_checks_run_on_the_host():
+    lib = api.lib()
+    n = C.c_size_t(0)
+
+    def code(**kw):
+        base = dict(P=4, M=4096, hidden=1024, ffn=2048, activation=api.ACT_SWIGLU)
+        base.update(kw)
+        return lib.compass_mlp_workspace_bytes(C.byref(api.make_mlp(**base)), C.byref(n))
+
+    assert code() == api.OK and n.value >= api.STATUS_BYTES
+    # the workspace serves both kernels: at least what each needs on its own
+    ag = api.make_problem(OP_AG_GEMM, 4, 4096, 2048, 1024)
+    rs = api.make_problem(OP_GEMM_RS, 4, 4096, 1024, 1024, rs_variant=api.RS_RING_RMW)
+    assert code(rs_variant=api.RS_RING_RMW) == api.OK
+    assert n.value == max(api.compass_workspace_bytes(ag, api.WS_FUSED), api.compass_workspace_bytes(rs, api.WS_FUSED))
+    assert lib.compass_mlp_workspace_bytes(None, C.byref(n)) == api.ERR_INVALID_ARG
+    assert lib.compass_mlp_workspace_bytes(C.byref(api.make_mlp(4, 4096, 1024, 2048)), None) == api.ERR_INVALID_ARG
+    assert code(activation=3) == api.ERR_INVALID_ARG
+    assert code(P=0) == api.ERR_INVALID_ARG
+    assert code(rings=3) == api.ERR_INVALID_ARG
+    assert code(rs_variant=5) == api.ERR_INVALID_ARG
+    assert code(P=3) == api.ERR_SHAPE                       # 4096 rows do not split over 3 ranks
+    assert code(hidden=0) == api.ERR_SHAPE
+    assert code(ffn=2056) == api.ERR_ALIGNMENT              # SwiGLU needs (gate, up) pairs and 16-byte rows of H
+    assert code(ffn=2056, activation=api.ACT_GELU_TANH) == api.OK
+    assert code(hidden=1020) == api.ERR_ALIGNMENT
+    assert code(P=32, M=8192) == api.ERR_UNSUPPORTED
+    bad = api.make_mlp(4, 4096, 1024, 2048)
+    bad.reserved = 1
+    assert lib.compass_mlp_workspace_bytes(C.byref(bad), C.byref(n)) == api.ERR_INVALID_ARG
+    # the block itself refuses NULL pointer arrays before any CUDA call
+    mp = api.make_mlp(4, 4096, 1024, 2048)
+    assert lib.compass_mlp_block(C.byref(mp), None, None, None, None, None, None, 0, None) == api.ERR_INVALID_ARG
+    assert lib.compass_mlp_block(None, None, None, None, None, None, None, 0, None) == api.ERR_INVALID_ARG
 
 
 def test_read_kernel_clock_rejects_null_arguments_before_touching_a_device():
