@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes (read + written) per launch of the GEMM kernel, from an ncu capture of
 # `bench.py --steps 1 --warmup 3 --no-cpu-baseline --no-sweep` (dram__bytes_read.sum + dram__bytes_write.sum).
-NCU_TRAFFIC_BYTES = {"C2": 360.4e6, "C3": 840.0e6}
+NCU_TRAFFIC_BYTES = {"C2": 362.6e6, "C3": 799.0e6}
 
 
 def env_int(name, default):
