@@ -90,6 +90,11 @@ enum { COMPASS_ORDER_RANK_MAJOR = 0, COMPASS_ORDER_STEP_MAJOR = 1 };
  * collective would be; it shares the SMs with the sub-GEMM it overlaps), or P*P device-to-device
  * copies per stage on the copy engines (no SM use, but P*P*d calls on the host). */
 enum { COMPASS_COPY_KERNEL = 0, COMPASS_COPY_ENGINES = 1 };
+/* Storage of the weight tensors B_r.  NK: [N][K], K contiguous (a linear layer's weight as the forward pass
+ * multiplies by it) -- the default.  KN: [K][N], N contiguous: the same stored weight used by the backward pass,
+ * where the data gradient multiplies by the transpose, so that AllGather+GEMM and GEMM+ReduceScatter of the
+ * backward pass run on the weights as they are, without a transposed copy. */
+enum { COMPASS_B_NK = 0, COMPASS_B_KN = 1 };
 /* selectors for compass_workspace_bytes */
 enum { COMPASS_WS_FUSED = 0, COMPASS_WS_DECOMP = 1, COMPASS_WS_PUSH = 2 };
 
@@ -105,6 +110,8 @@ typedef struct compass_problem {
   int32_t rs_variant;  /* COMPASS_RS_* (GEMM+ReduceScatter only) */
   int32_t order;       /* COMPASS_ORDER_* : how the P logical ranks share the one GPU */
   int32_t copy_mode;   /* COMPASS_COPY_* : how compass_decomp moves the AllGather slices */
+  int32_t b_layout;    /* COMPASS_B_* : storage of every B_r */
+  int32_t reserved;    /* 0 */
 } compass_problem;
 
 /* One line of the ring chunk schedule (Section III-B).  `part` = rings*chunk +
@@ -248,7 +255,12 @@ int compass_select(const compass_problem* problem, const compass_calib* calib, c
  *   Out: P device pointers, Out[r] = [M/P x hidden]
  *   workspace: >= compass_mlp_workspace_bytes bytes, 256-byte aligned, zeroed
  *   once with compass_workspace_init; compass_read_status reports a bounded
- *   wait of either kernel that gave up. */
+ *   wait of either kernel that gave up.
+ * Backward pass: the data gradients of the literal block (no activation) are
+ * the same chain run on the stored weights with COMPASS_B_KN --
+ * dH_r = gather(dOut) * W1_r and dX_c = rows of sum_q dH_q * W0_q, i.e. the
+ * call (dOut, W1, dH, W0, dX) with hidden and ffn unchanged.  Activation
+ * derivatives and weight gradients are not part of this library. */
 enum { COMPASS_ACT_NONE = 0, COMPASS_ACT_GELU_TANH = 1, COMPASS_ACT_SWIGLU = 2 };
 typedef struct compass_mlp {
   int32_t P;           /* tensor-parallel size */
@@ -259,7 +271,7 @@ typedef struct compass_mlp {
   int32_t activation;  /* COMPASS_ACT_* */
   int32_t rs_variant;  /* COMPASS_RS_* of the second kernel */
   int32_t order;       /* COMPASS_ORDER_* of the first kernel */
-  int32_t reserved;    /* 0 */
+  int32_t b_layout;    /* COMPASS_B_* : storage of W0_r and W1_r (KN: [hidden x ffn] and [hc x hidden]) */
 } compass_mlp;
 int compass_mlp_workspace_bytes(const compass_mlp* mlp, size_t* bytes);
 int compass_mlp_block(const compass_mlp* mlp, const void* const* X, const void* const* W0, void* const* H,

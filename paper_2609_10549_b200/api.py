@@ -26,6 +26,7 @@ ORDER_RANK_MAJOR, ORDER_STEP_MAJOR = 0, 1
 COPY_KERNEL, COPY_ENGINES = 0, 1
 WS_FUSED, WS_DECOMP, WS_PUSH = 0, 1, 2
 ACT_NONE, ACT_GELU_TANH, ACT_SWIGLU = 0, 1, 2
+B_NK, B_KN = 0, 1
 MAX_P = 16
 STATUS_BYTES = 256
 
@@ -50,12 +51,13 @@ class CompassError(RuntimeError):
 class Problem(C.Structure):
     _fields_ = [("op", C.c_int32), ("P", C.c_int32), ("rings", C.c_int32), ("d", C.c_int32),
                 ("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64),
-                ("dtype", C.c_int32), ("rs_variant", C.c_int32), ("order", C.c_int32), ("copy_mode", C.c_int32)]
+                ("dtype", C.c_int32), ("rs_variant", C.c_int32), ("order", C.c_int32), ("copy_mode", C.c_int32),
+                ("b_layout", C.c_int32), ("reserved", C.c_int32)]
 
 
 class Mlp(C.Structure):
     _fields_ = [("P", C.c_int32), ("rings", C.c_int32), ("M", C.c_int64), ("hidden", C.c_int64), ("ffn", C.c_int64),
-                ("activation", C.c_int32), ("rs_variant", C.c_int32), ("order", C.c_int32), ("reserved", C.c_int32)]
+                ("activation", C.c_int32), ("rs_variant", C.c_int32), ("order", C.c_int32), ("b_layout", C.c_int32)]
 
 
 class SchedEntry(C.Structure):
@@ -146,9 +148,9 @@ def _check(status: int, where: str) -> None:
 
 def make_problem(op: int, P: int, M: int, N: int, K: int, rings: int = 2, d: int = 1,
                  rs_variant: int = RS_SEGMENTED_K, dtype: int = DTYPE_BF16, order: int = ORDER_RANK_MAJOR,
-                 copy_mode: int = COPY_KERNEL) -> Problem:
+                 copy_mode: int = COPY_KERNEL, b_layout: int = B_NK) -> Problem:
     return Problem(op=op, P=P, rings=rings, d=d, M=M, N=N, K=K, dtype=dtype, rs_variant=rs_variant, order=order,
-                   copy_mode=copy_mode)
+                   copy_mode=copy_mode, b_layout=b_layout, reserved=0)
 
 
 # ---- host-only calls -------------------------------------------------------------
@@ -291,9 +293,9 @@ def compass_ag_gemm_push(problem: Problem, A: Sequence, B: Sequence, Cout: Seque
 
 
 def make_mlp(P: int, M: int, hidden: int, ffn: int, activation: int = 0, rings: int = 2,
-             rs_variant: int = RS_SEGMENTED_K, order: int = ORDER_RANK_MAJOR) -> Mlp:
+             rs_variant: int = RS_SEGMENTED_K, order: int = ORDER_RANK_MAJOR, b_layout: int = B_NK) -> Mlp:
     return Mlp(P=P, rings=rings, M=M, hidden=hidden, ffn=ffn, activation=activation, rs_variant=rs_variant,
-               order=order, reserved=0)
+               order=order, b_layout=b_layout)
 
 
 def compass_mlp_workspace_bytes(mlp: Mlp) -> int:

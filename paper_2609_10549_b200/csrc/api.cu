@@ -29,6 +29,7 @@ int validate_problem(const compass_problem* pr, int want_op, bool need_d) {
   if (pr->copy_mode != COMPASS_COPY_KERNEL && pr->copy_mode != COMPASS_COPY_ENGINES) return COMPASS_ERR_INVALID_ARG;
   if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant != COMPASS_RS_SEGMENTED_K && pr->rs_variant != COMPASS_RS_RING_RMW)
     return COMPASS_ERR_INVALID_ARG;
+  if ((pr->b_layout != COMPASS_B_NK && pr->b_layout != COMPASS_B_KN) || pr->reserved != 0) return COMPASS_ERR_INVALID_ARG;
   if (pr->dtype != COMPASS_DTYPE_BF16 || pr->P > COMPASS_MAX_P) return COMPASS_ERR_UNSUPPORTED;
   if (pr->M <= 0 || pr->N <= 0 || pr->K <= 0) return COMPASS_ERR_SHAPE;
   if (pr->M % pr->P != 0 || (pr->M / pr->P) % pr->rings != 0) return COMPASS_ERR_SHAPE;
@@ -204,6 +205,7 @@ int plan_fused(const compass_problem* pr, GemmLaunch* L, compass_plan_block* vie
   if (pr->op == COMPASS_OP_AG_GEMM) plan_ag(pr, table, L, view);
   else if (pr->rs_variant == COMPASS_RS_SEGMENTED_K) plan_rs_segmented(pr, table, L, view);
   else plan_rs_ring(pr, table, L, view);
+  L->b_mn_major = pr->b_layout == COMPASS_B_KN;
   if (view) {
     const int per_block = tiles_of(L->rows_per_block, gemm_tile_rows(L->mode, L->rows_per_block)) * tiles_of(L->N, BN);
     for (int i = 0; i < L->n_blocks; ++i) {
@@ -242,7 +244,7 @@ int mlp_problems(const compass_mlp* mp, compass_problem* ag, compass_problem* rs
   if (mp == nullptr) return COMPASS_ERR_INVALID_ARG;
   if (mp->activation != COMPASS_ACT_NONE && mp->activation != COMPASS_ACT_GELU_TANH && mp->activation != COMPASS_ACT_SWIGLU)
     return COMPASS_ERR_INVALID_ARG;
-  if (mp->reserved != 0) return COMPASS_ERR_INVALID_ARG;
+  if (mp->b_layout != COMPASS_B_NK && mp->b_layout != COMPASS_B_KN) return COMPASS_ERR_INVALID_ARG;
   if (mp->hidden <= 0 || mp->ffn <= 0) return COMPASS_ERR_SHAPE;
   // SwiGLU: (gate, up) column pairs; the result's rows must still be a multiple of 16 bytes for the second GEMM's loads
   if (mp->activation == COMPASS_ACT_SWIGLU && mp->ffn % 16 != 0) return COMPASS_ERR_ALIGNMENT;
@@ -258,6 +260,7 @@ int mlp_problems(const compass_mlp* mp, compass_problem* ag, compass_problem* rs
   ag->rs_variant = COMPASS_RS_SEGMENTED_K;
   ag->order = mp->order;
   ag->copy_mode = COMPASS_COPY_KERNEL;
+  ag->b_layout = mp->b_layout;
   *rs = *ag;
   rs->op = COMPASS_OP_GEMM_RS;
   rs->N = mp->hidden;
@@ -305,6 +308,7 @@ int decomp_ag(const compass_problem* pr, const void* const* A, const void* const
 
   static thread_local GemmLaunch L;
   L.n_a = L.n_b = L.n_out = P;
+  L.b_mn_major = pr->b_layout == COMPASS_B_KN;
   L.a_rows = pr->M;
   L.K = K;
   L.N = pr->N;
@@ -370,6 +374,7 @@ int decomp_rs(const compass_problem* pr, const void* const* A, const void* const
 
   static thread_local GemmLaunch L;
   L.n_a = L.n_b = L.n_out = P;
+  L.b_mn_major = pr->b_layout == COMPASS_B_KN;
   L.a_rows = pr->M;
   L.K = pr->K;
   L.N = pr->N;
@@ -608,6 +613,7 @@ extern "C" int compass_ag_gemm_push(const compass_problem* pr, const void* const
 
   static thread_local GemmLaunch L;
   L.n_a = 2 * P;                       // maps 0..P-1: the shards, P..2P-1: the gather buffers
+  L.b_mn_major = pr->b_layout == COMPASS_B_KN;
   L.n_b = L.n_out = P;
   L.a_rows = m;
   L.K = K;

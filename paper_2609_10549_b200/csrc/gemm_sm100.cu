@@ -66,6 +66,9 @@ struct Cfg {
   static constexpr uint32_t kFullTxBytes = kPair ? 2 * kStageBytes : kStageBytes;
 };
 
+// An N-contiguous B tile is kept as chunks of 64 columns x 64 k-rows (what one tensor-map box of 128-byte rows holds).
+constexpr int kBChunkMnBytes = 64 * BK * 2;
+
 struct Control {
   uint64_t full[kSlots];
   uint64_t empty[kSlots];
@@ -308,8 +311,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
           for (int at = 0; at < C::kAtoms; ++at) {
             tma_load_2d_pair_hint(smem_a + stage * C::kATileBytes + at * C::kAAtomBytes, &p.a_maps[ld.am], full_addr,
                                   kx + at * BK, ld.a_row, pol_a);
-            tma_load_2d_pair_hint(smem_b + stage * C::kBTileBytes + at * C::kBAtomBytes, &p.b_maps[ld.bm], full_addr,
-                                  kx + at * BK, ld.b_row, pol_b);
+            uint8_t* b_dst = smem_b + stage * C::kBTileBytes + at * C::kBAtomBytes;
+            if (p.b_mn_major) {
+              // B is [K][N]: boxes of 64 columns (N) x 64 rows (K), one 8 KB chunk per 64 columns
+#pragma unroll
+              for (int ch = 0; ch < C::kBRows / 64; ++ch)
+                tma_load_2d_pair_hint(b_dst + ch * kBChunkMnBytes, &p.b_maps[ld.bm], full_addr, ld.b_row + ch * 64, kx + at * BK, pol_b);
+            } else {
+              tma_load_2d_pair_hint(b_dst, &p.b_maps[ld.bm], full_addr, kx + at * BK, ld.b_row, pol_b);
+            }
           }
         } else {
           mbar_arrive_expect_tx(&ctl->full[stage], C::kFullTxBytes);
@@ -317,11 +327,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
           for (int at = 0; at < C::kAtoms; ++at) {
             tma_load_2d_hint(smem_a + stage * C::kATileBytes + at * C::kAAtomBytes, &p.a_maps[ld.am], &ctl->full[stage],
                              kx + at * BK, ld.a_row, pol_a);
-            tma_load_2d_hint(smem_b + stage * C::kBTileBytes + at * C::kBAtomBytes, &p.b_maps[ld.bm], &ctl->full[stage],
-                             kx + at * BK, ld.b_row, pol_b);
+            uint8_t* b_dst = smem_b + stage * C::kBTileBytes + at * C::kBAtomBytes;
+            if (p.b_mn_major) {
+#pragma unroll
+              for (int ch = 0; ch < C::kBRows / 64; ++ch)
+                tma_load_2d_hint(b_dst + ch * kBChunkMnBytes, &p.b_maps[ld.bm], &ctl->full[stage], ld.b_row + ch * 64, kx + at * BK, pol_b);
+            } else {
+              tma_load_2d_hint(b_dst, &p.b_maps[ld.bm], &ctl->full[stage], kx + at * BK, ld.b_row, pol_b);
+            }
           }
         }
-        if (p.prefetch_stages > 0 && pf.valid(p)) {
+        if (p.prefetch_stages > 0 && !p.b_mn_major && pf.valid(p)) {
           const int px = pf.kb * C::kStageK;
 #pragma unroll
           for (int at = 0; at < C::kAtoms; ++at) {
@@ -356,10 +372,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     // One lane runs the whole loop (a per-instruction "if (lane == 0)" inside a
     // 32-lane loop costs a divergence per MMA and slows the issue stream).
     if (leader && lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16_f32(kPair ? 2 * BM : BM, BN);
+      const uint32_t idesc = umma_idesc_bf16_f32(kPair ? 2 * BM : BM, BN) | (p.b_mn_major ? kUmmaIdescBMnMajor : 0u);
       constexpr int kFullSteps = C::kStageK / UMMA_K;
       const uint64_t desc_a0 = umma_smem_desc_sw128(smem_u32(smem_a));
-      const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(smem_b));
+      const uint64_t desc_b0 = p.b_mn_major ? umma_smem_desc_sw128_mn(smem_u32(smem_b), kBChunkMnBytes)
+                                            : umma_smem_desc_sw128(smem_u32(smem_b));
+      // address-field step per 16-element k-step: 32 bytes inside a K-major swizzle row, two 8-row groups
+      // (2048 bytes) in an N-contiguous chunk
+      const uint32_t b_kstep = p.b_mn_major ? (2 * 1024) >> 4 : 2;
       int stage = 0;
       uint32_t phase = 0;
       uint32_t it = 0;
@@ -386,14 +406,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             for (int ks = 0; ks < kFullSteps; ++ks) {
               // a 64-element atom holds 4 steps of 16 elements = 32 bytes each: +2 in the address field
               const uint64_t a_k = da + uint64_t(((ks >> 2) * C::kAAtomBytes >> 4) + (ks & 3) * 2);
-              const uint64_t b_k = db + uint64_t(((ks >> 2) * C::kBAtomBytes >> 4) + (ks & 3) * 2);
+              const uint64_t b_k = db + uint64_t(((ks >> 2) * C::kBAtomBytes >> 4) + (ks & 3) * b_kstep);
               if (kPair) umma_bf16_pair(d_tmem, a_k, b_k, idesc, ks ? 1u : first);
               else umma_bf16(d_tmem, a_k, b_k, idesc, ks ? 1u : first);
             }
           } else {
             for (int ks = 0; ks < p.tail_ksteps; ++ks) {
               const uint64_t a_k = da + uint64_t(((ks >> 2) * C::kAAtomBytes >> 4) + (ks & 3) * 2);
-              const uint64_t b_k = db + uint64_t(((ks >> 2) * C::kBAtomBytes >> 4) + (ks & 3) * 2);
+              const uint64_t b_k = db + uint64_t(((ks >> 2) * C::kBAtomBytes >> 4) + (ks & 3) * b_kstep);
               if (kPair) umma_bf16_pair(d_tmem, a_k, b_k, idesc, ks ? 1u : first);
               else umma_bf16(d_tmem, a_k, b_k, idesc, ks ? 1u : first);
             }
@@ -711,18 +731,28 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
         uint8_t* c0 = smem + ((chunk + 0) % kChunks) * kChunkBytes;
         uint8_t* c1 = smem + ((chunk + 1) % kChunks) * kChunkBytes;
         uint8_t* c2 = smem + ((chunk + 2) % kChunks) * kChunkBytes;
+        // this CTA's 128 rows of B for one 64-wide k-atom: one box when B is [N][K], two boxes of 64 columns
+        // (8 KB chunks) when B is [K][N]
+        auto load_b = [&](uint8_t* dst, int kx) {
+          if (p.b_mn_major) {
+            tma_load_2d_pair_hint(dst, &p.b_maps[it.bm], full_addr, it.b_row, kx, pol_b);
+            tma_load_2d_pair_hint(dst + kBChunkMnBytes, &p.b_maps[it.bm], full_addr, it.b_row + 64, kx, pol_b);
+          } else {
+            tma_load_2d_pair_hint(dst, &p.b_maps[it.bm], full_addr, kx, it.b_row, pol_b);
+          }
+        };
         if (big) {
           const int kx = it.kb * BK;
           tma_load_2d_pair_hint(c0, &p.a_maps[it.am], full_addr, kx, it.a_row, pol_a);
           tma_load_2d_pair_hint(c1, &p.a_maps[it.am], full_addr, kx, it.a_row + BM, pol_a);
-          tma_load_2d_pair_hint(c2, &p.b_maps[it.bm], full_addr, kx, it.b_row, pol_b);
+          load_b(c2, kx);
         } else {
           const int kx = it.kb * 2 * BK;
           uint8_t* c3 = smem + ((chunk + 3) % kChunks) * kChunkBytes;
           tma_load_2d_pair_hint(c0, &p.a_maps[it.am], full_addr, kx, it.a_row, pol_a);
-          tma_load_2d_pair_hint(c2, &p.b_maps[it.bm], full_addr, kx, it.b_row, pol_b);
+          load_b(c2, kx);
           tma_load_2d_pair_hint(c1, &p.a_maps[it.am], full_addr, kx + BK, it.a_row, pol_a);
-          tma_load_2d_pair_hint(c3, &p.b_maps[it.bm], full_addr, kx + BK, it.b_row, pol_b);
+          load_b(c3, kx + BK);
         }
         chunk = (chunk + nchunks) % kChunks;
       }
@@ -738,8 +768,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
     // One lane runs the whole loop: a per-instruction "if (lane == 0)" inside a
     // 32-lane loop costs a divergence per MMA and measurably slows the issue stream.
     if (leader && lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16_f32(2 * BM, BN);
+      const uint32_t idesc = umma_idesc_bf16_f32(2 * BM, BN) | (p.b_mn_major ? kUmmaIdescBMnMajor : 0u);
       const uint64_t desc0 = umma_smem_desc_sw128(smem_u32(smem));
+      // B chunks: the same ring, but an N-contiguous chunk is two 8 KB sub-chunks and a k-step is 2048 bytes
+      const uint64_t desc0b = p.b_mn_major ? umma_smem_desc_sw128_mn(smem_u32(smem), kBChunkMnBytes) : desc0;
+      const uint32_t bk = p.b_mn_major ? (2 * 1024) >> 4 : 2;
       uint32_t j = 0;
       int chunk = 0;
       uint32_t uses0 = 0, uses1 = 0;      // completed uses of accumulator 0 / 1
@@ -768,12 +801,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
           auto ksteps = [&](int kb) { return (kb % kb_seg == kb_seg - 1) ? tail : BK / UMMA_K; };
           auto issue = [&](uint32_t acc, int a_chunk, int b_chunk, int nk, uint32_t first) {
             const uint64_t da = desc0 + uint64_t(((a_chunk % kChunks) * kChunkBytes) >> 4);
-            const uint64_t db = desc0 + uint64_t(((b_chunk % kChunks) * kChunkBytes) >> 4);
+            const uint64_t db = desc0b + uint64_t(((b_chunk % kChunks) * kChunkBytes) >> 4);
             if (nk == BK / UMMA_K) {
 #pragma unroll
-              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc, da + uint64_t(k * 2), db + uint64_t(k * 2), idesc, k ? 1u : first);
+              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc, da + uint64_t(k * 2), db + uint64_t(k * bk), idesc, k ? 1u : first);
             } else {
-              for (int k = 0; k < nk; ++k) umma_bf16_pair(acc, da + uint64_t(k * 2), db + uint64_t(k * 2), idesc, k ? 1u : first);
+              for (int k = 0; k < nk; ++k) umma_bf16_pair(acc, da + uint64_t(k * 2), db + uint64_t(k * bk), idesc, k ? 1u : first);
             }
           };
           // `count` stages from stage kb on, accumulator 0 first, then accumulator 1 (which releases the stages)
@@ -813,19 +846,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
             tc_fence_after_sync();
             const uint64_t d0 = desc0 + uint64_t((((chunk + 0) % kChunks) * kChunkBytes) >> 4);
             const uint64_t d1 = desc0 + uint64_t((((chunk + 1) % kChunks) * kChunkBytes) >> 4);
-            const uint64_t d2 = desc0 + uint64_t((((chunk + 2) % kChunks) * kChunkBytes) >> 4);
+            const uint64_t d2 = desc0b + uint64_t((((chunk + 2) % kChunks) * kChunkBytes) >> 4);
             const uint32_t first = kb != 0 ? 1u : 0u;
             const int nk = ksteps(kb);
             if (nk == BK / UMMA_K) {
 #pragma unroll
               for (int k = 0; k < BK / UMMA_K; ++k) {
-                umma_bf16_pair(tmem_base, d0 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
-                umma_bf16_pair(tmem_base + BN, d1 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
+                umma_bf16_pair(tmem_base, d0 + uint64_t(k * 2), d2 + uint64_t(k * bk), idesc, k ? 1u : first);
+                umma_bf16_pair(tmem_base + BN, d1 + uint64_t(k * 2), d2 + uint64_t(k * bk), idesc, k ? 1u : first);
               }
             } else {
               for (int k = 0; k < nk; ++k) {
-                umma_bf16_pair(tmem_base, d0 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
-                umma_bf16_pair(tmem_base + BN, d1 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
+                umma_bf16_pair(tmem_base, d0 + uint64_t(k * 2), d2 + uint64_t(k * bk), idesc, k ? 1u : first);
+                umma_bf16_pair(tmem_base + BN, d1 + uint64_t(k * 2), d2 + uint64_t(k * bk), idesc, k ? 1u : first);
               }
             }
             chunk = (chunk + 3) % kChunks;
@@ -852,18 +885,18 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
             const bool full_stage = kb_in_seg != kb_seg - 1 || tail == 2 * BK / UMMA_K;
             const uint64_t d0 = desc0 + uint64_t((((chunk + 0) % kChunks) * kChunkBytes) >> 4);
             const uint64_t d1 = desc0 + uint64_t((((chunk + 1) % kChunks) * kChunkBytes) >> 4);
-            const uint64_t d2 = desc0 + uint64_t((((chunk + 2) % kChunks) * kChunkBytes) >> 4);
-            const uint64_t d3 = desc0 + uint64_t((((chunk + 3) % kChunks) * kChunkBytes) >> 4);
+            const uint64_t d2 = desc0b + uint64_t((((chunk + 2) % kChunks) * kChunkBytes) >> 4);
+            const uint64_t d3 = desc0b + uint64_t((((chunk + 3) % kChunks) * kChunkBytes) >> 4);
             const uint32_t first = kb != 0 ? 1u : 0u;
             if (full_stage) {
 #pragma unroll
-              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc_a, d0 + uint64_t(k * 2), d2 + uint64_t(k * 2), idesc, k ? 1u : first);
+              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc_a, d0 + uint64_t(k * 2), d2 + uint64_t(k * bk), idesc, k ? 1u : first);
 #pragma unroll
-              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc_a, d1 + uint64_t(k * 2), d3 + uint64_t(k * 2), idesc, 1u);
+              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc_a, d1 + uint64_t(k * 2), d3 + uint64_t(k * bk), idesc, 1u);
             } else {
               for (int ks = 0; ks < tail; ++ks) {
                 const int k = ks & 3;
-                umma_bf16_pair(acc_a, ((ks >> 2) ? d1 : d0) + uint64_t(k * 2), ((ks >> 2) ? d3 : d2) + uint64_t(k * 2), idesc,
+                umma_bf16_pair(acc_a, ((ks >> 2) ? d1 : d0) + uint64_t(k * 2), ((ks >> 2) ? d3 : d2) + uint64_t(k * bk), idesc,
                                ks ? 1u : first);
               }
             }
@@ -1108,7 +1141,9 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
     if (!encode_kmajor(&p.a_maps[i], L.a_ptr[i], L.a_map_rows[i] ? L.a_map_rows[i] : L.a_rows, L.K, BM))
       return record_cuda_error(cudaErrorUnknown);
   for (int i = 0; i < L.n_b; ++i)
-    if (!encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, b_box_rows)) return record_cuda_error(cudaErrorUnknown);
+    if (L.b_mn_major ? !encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.K, L.N, 64)      // [K][N]: boxes of 64 columns x 64 k-rows
+                     : !encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, b_box_rows))
+      return record_cuda_error(cudaErrorUnknown);
   for (int i = 0; i < L.n_out; ++i) p.out[i] = static_cast<__nv_bfloat16*>(L.out_ptr[i]);
   p.ldo = L.ldo;
   p.n_blocks = L.n_blocks;
@@ -1127,6 +1162,7 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   p.wait_limit_us = L.wait_limit_us ? L.wait_limit_us : (default_wait_limit_us() ? default_wait_limit_us() : 2000000u);
   p.prefetch_stages = L.prefetch_stages;
   p.activation = L.activation;
+  p.b_mn_major = L.b_mn_major ? 1 : 0;
   p.skew = L.skew < 0 ? 0 : (L.skew > 4 ? 4 : L.skew);
   p.a_hint = L.a_hint;
   p.b_hint = L.b_hint;
@@ -1181,7 +1217,7 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
       p.kb_per_seg = int32_t((L.K + BK - 1) / BK);
       p.tail_ksteps = int32_t((L.K - int64_t(p.kb_per_seg - 1) * BK + UMMA_K - 1) / UMMA_K);
       for (int i = 0; i < L.n_b; ++i)
-        if (!encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, BN)) return record_cuda_error(cudaErrorUnknown);
+        if (!L.b_mn_major && !encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, BN)) return record_cuda_error(cudaErrorUnknown);
     }
     const int grid = p.total_tiles < info->num_sms ? p.total_tiles : info->num_sms;
     if (L.activation != ACT_NONE) gemm_kernel<false, true><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);

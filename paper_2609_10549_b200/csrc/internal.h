@@ -97,6 +97,7 @@ struct GemmParams {
   uint32_t wait_limit_us;  // bound of every device-side wait
   int32_t a_hint, b_hint;  // L2 eviction priority of the A / B tile loads (ptx::L2Hint)
   int32_t prefetch_stages; // how many k-stages ahead of the shared-memory loads operands are prefetched into L2 (0 = off)
+  int32_t b_mn_major;      // 1: the B tensors are stored [K][N] (N contiguous); 0: [N][K]
   int32_t activation;      // ActivationMode applied to the FP32 accumulator before the BF16 store (plain-store epilogue only)
   int32_t skew;            // 512x256 tiles: stages at each end of a tile in which accumulator 0 runs ahead of accumulator 1 (0..4)
   StatusBlock* status;
@@ -126,6 +127,7 @@ struct GemmLaunch {
   int b_hint = 2;   // weight tiles: evict last (measured 1-2 % shorter kernels than the default priority)
   int prefetch_stages = 0;
   int activation = 0;   // ActivationMode
+  int b_mn_major = 0;   // 1: B tensors are [K][N]
   int skew = 3;     // 512x256 tiles: stages at each end of a tile with accumulator 0 ahead of accumulator 1 (measured: 3 of 0..4)
   uint32_t wait_limit_us = 0;   // 0 = default bound of the device-side waits
   int last_step = 0;

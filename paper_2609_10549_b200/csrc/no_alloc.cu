@@ -91,6 +91,7 @@ extern "C" int compass_gemm_rs_sequential_noalloc(const compass_problem* pr, con
 
   static thread_local GemmLaunch L;
   L.n_a = L.n_b = L.n_out = P;
+  L.b_mn_major = pr->b_layout == COMPASS_B_KN;
   L.a_rows = pr->M;
   L.K = pr->K;
   L.N = pr->N;

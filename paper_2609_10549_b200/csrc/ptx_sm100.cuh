@@ -134,12 +134,22 @@ __device__ __forceinline__ uint64_t umma_smem_desc_sw128(uint32_t smem_addr) {
   return d;
 }
 
+// The same for an MN-major operand tile with 128-byte swizzle: the tile is a row of chunks, each chunk
+// 64 MN-elements (128 bytes) wide and stored as consecutive K rows of 128 bytes, swizzled in groups of
+// 8 rows (1024 bytes).  SBO = distance between 8-row K groups (1024), LBO = distance between chunks.
+__device__ __forceinline__ uint64_t umma_smem_desc_sw128_mn(uint32_t smem_addr, uint32_t chunk_bytes) {
+  uint64_t d = umma_smem_desc_sw128(smem_addr);
+  d |= static_cast<uint64_t>(chunk_bytes >> 4) << 16;
+  return d;
+}
+
 // Instruction descriptor for kind::f16 with BF16 A and B (both K-major), FP32
 // accumulator.  Bits: [4,6) D format (1 = F32), [7,10) A format (1 = BF16),
 // [10,13) B format, 15/16 A/B major (0 = K), [17,23) N>>3, [24,29) M>>4.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(uint32_t m, uint32_t n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((m >> 4) << 24);
 }
+constexpr uint32_t kUmmaIdescBMnMajor = 1u << 16;      // B operand stored with N contiguous
 
 // D[tmem] (+)= A[smem] * B[smem]; issued by ONE thread.
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {

@@ -30,7 +30,8 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_layouts_match_the_header():
-    assert C.sizeof(api.Problem) == 4 * 4 + 3 * 8 + 4 * 4
+    assert C.sizeof(api.Problem) == 4 * 4 + 3 * 8 + 6 * 4
+    assert api.Problem.b_layout.offset == 56
     assert C.sizeof(api.SchedEntry) == 32
     assert C.sizeof(api.Calib) == 64
     assert C.sizeof(api.Choice) == 8 + 6 * 8
@@ -152,9 +153,8 @@ def test_mlp_block_argument_checks_run_on_the_host():
     assert code(ffn=2056, activation=api.ACT_GELU_TANH) == api.OK
     assert code(hidden=1020) == api.ERR_ALIGNMENT
     assert code(P=32, M=8192) == api.ERR_UNSUPPORTED
-    bad = api.make_mlp(4, 4096, 1024, 2048)
-    bad.reserved = 1
-    assert lib.compass_mlp_workspace_bytes(C.byref(bad), C.byref(n)) == api.ERR_INVALID_ARG
+    assert code(b_layout=api.B_KN) == api.OK
+    assert code(b_layout=2) == api.ERR_INVALID_ARG
     # the block itself refuses NULL pointer arrays before any CUDA call
     mp = api.make_mlp(4, 4096, 1024, 2048)
     assert lib.compass_mlp_block(C.byref(mp), None, None, None, None, None, None, 0, None) == api.ERR_INVALID_ARG
@@ -202,6 +202,11 @@ def test_problem_validation_codes():
     ok = dict(op=OP_AG_GEMM, P=4, M=4096, N=3072, K=4096)
     assert _codes(api.make_problem(**ok))[0] == api.OK
     assert _codes(api.make_problem(**{**ok, "op": 9}))[0] == api.ERR_INVALID_ARG
+    assert _codes(api.make_problem(**{**ok, "b_layout": api.B_KN}))[0] == api.OK
+    assert _codes(api.make_problem(**{**ok, "b_layout": 2}))[0] == api.ERR_INVALID_ARG
+    nonzero_reserved = api.make_problem(**ok)
+    nonzero_reserved.reserved = 1
+    assert _codes(nonzero_reserved)[0] == api.ERR_INVALID_ARG
     assert _codes(api.make_problem(**{**ok, "P": 0}))[0] == api.ERR_INVALID_ARG
     assert _codes(api.make_problem(**ok, rings=3))[0] == api.ERR_INVALID_ARG
     assert _codes(api.make_problem(**{**ok, "P": 32, "M": 4096}))[0] == api.ERR_UNSUPPORTED

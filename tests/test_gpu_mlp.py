@@ -144,3 +144,46 @@ def test_mlp_block_repeated_calls_are_bitwise_identical():
     b = run_block(P, m, hidden, ffn, act, X, W0, W1, hc)
     for x, y in zip(a[0] + a[1], b[0] + b[1]):
         assert (x == y).all()
+
+
+def test_backward_data_gradients_are_the_block_on_the_stored_weights():
+    """dH_r = gather(dOut) * W1_r and dX = ReduceScatter(sum_q dH_q * W0_q): the block itself, called with
+    the weights as stored ([hidden x hc] and [ffn x hidden]) and the [K][N] layout flag."""
+    P, m, hidden, ffn = 4, 512, 264, 1040
+    w = wl.MlpWorkload("mlp-bwd", P=P, M=P * m, hidden=hidden, ffn=ffn, activation=omlp.ACT_NONE, seed=5)
+    dOut, W0, W1 = wl.make_mlp_inputs(w)                     # dOut_r [m x hidden], W0_r [ffn x hidden], W1_r [hidden x ffn]
+    mp = api.make_mlp(P, P * m, hidden, ffn, activation=api.ACT_NONE, b_layout=api.B_KN)
+    d_dOut, dW0, dW1 = [api.to_device(a) for a in dOut], [api.to_device(a) for a in W0], [api.to_device(a) for a in W1]
+    dH = [gu.Guarded(P * m, ffn) for _ in range(P)]
+    dX = [gu.Guarded(m, hidden) for _ in range(P)]
+    ws = api.alloc_mlp_workspace(mp)
+    api.compass_mlp_block(mp, d_dOut, dW1, [t.view for t in dH], dW0, [t.view for t in dX], ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    assert all(t.guards_intact() for t in dH + dX)
+    # oracle: the same chain with the weights written the way its GEMMs take them ([N][K])
+    W1_t = [np.ascontiguousarray(a.T) for a in W1]            # [ffn x hidden]
+    W0_t = [np.ascontiguousarray(a.T) for a in W0]            # [hidden x ffn]
+    dX_ref, dH_ref_bits = omlp.mlp_block(dOut, W1_t, W0_t, omlp.ACT_NONE)
+    C = ops.ag_gemm(dOut, W1_t)
+    for r in range(P):
+        rep = compare.check(dH[r].bits(), C[r])
+        assert rep.ok, f"dH rank {r}: {rep}"
+        rep = compare.check(dX[r].bits(), dX_ref[r])
+        assert rep.ok, f"dX rank {r}: {rep}"
+
+
+def test_mlp_block_kn_weights_match_nk_weights_bitwise():
+    P, m, hidden, ffn, act = 4, 512, 256, 1056, omlp.ACT_SWIGLU
+    X, W0, W1, hc = make_inputs(P, m, hidden, ffn, act)
+    nk = run_block(P, m, hidden, ffn, act, X, W0, W1, hc)
+    mp = api.make_mlp(P, P * m, hidden, ffn, activation=act, b_layout=api.B_KN)
+    dX = [api.to_device(a) for a in X]
+    dW0 = [api.to_device(np.ascontiguousarray(a.T)) for a in W0]
+    dW1 = [api.to_device(np.ascontiguousarray(a.T)) for a in W1]
+    H = [gu.Guarded(P * m, hc) for _ in range(P)]
+    Out = [gu.Guarded(m, hidden) for _ in range(P)]
+    ws = api.alloc_mlp_workspace(mp)
+    api.compass_mlp_block(mp, dX, dW0, [h.view for h in H], dW1, [o.view for o in Out], ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    for got, want in zip([h.bits() for h in H] + [o.bits() for o in Out], nk[0] + nk[1]):
+        assert (got == want).all()

@@ -413,3 +413,78 @@ def test_single_ring_and_double_ring_agree_bitwise_for_ag_gemm():
     one, _, _ = gu.run_fused(w, A, B, rings=1)
     for x, y in zip(one, two):
         assert np.array_equal(x, y)
+
+
+# ---- weights stored [K][N] (N contiguous): the layout the backward pass finds them in -----------------
+
+def run_with_kn_weights(w, A_bits, B_bits, rings=2, rs_variant=api.RS_SEGMENTED_K, order=api.ORDER_RANK_MAJOR):
+    pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, rings=rings, rs_variant=rs_variant, order=order, b_layout=api.B_KN)
+    A = [api.to_device(a) for a in A_bits]
+    B = [api.to_device(np.ascontiguousarray(b.T)) for b in B_bits]        # the same values, stored [K][N]
+    outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    ws = api.alloc_workspace(pr)
+    (api.compass_ag_gemm if w.op == wl.OP_AG_GEMM else api.compass_gemm_rs)(pr, A, B, [o.view for o in outs], ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    assert all(o.guards_intact() for o in outs)
+    return [o.bits() for o in outs]
+
+
+@pytest.mark.parametrize("op,P,m,N,K,rings", [
+    (wl.OP_AG_GEMM, 1, 128, 256, 64, 2), (wl.OP_AG_GEMM, 2, 256, 256, 256, 2), (wl.OP_AG_GEMM, 2, 144, 264, 72, 2),
+    (wl.OP_AG_GEMM, 3, 272, 520, 1376, 2), (wl.OP_AG_GEMM, 4, 384, 1024, 320, 1), (wl.OP_AG_GEMM, 8, 80, 200, 8, 2),
+    (wl.OP_GEMM_RS, 2, 256, 256, 256, 2), (wl.OP_GEMM_RS, 3, 272, 520, 344, 2), (wl.OP_GEMM_RS, 8, 256, 512, 1376, 2),
+    (wl.OP_GEMM_RS, 4, 384, 1024, 320, 1),
+])
+def test_kn_weights_small_shapes(op, P, m, N, K, rings):
+    w = small(op, P, m, N, K)
+    A, B = wl.make_inputs(w)
+    outs = run_with_kn_weights(w, A, B, rings=rings)
+    check_all(outs, ops.ag_gemm(A, B, rings=rings) if op == wl.OP_AG_GEMM else ops.gemm_rs(A, B, rings=rings), w.name)
+
+
+@pytest.mark.parametrize("op,P,m,N,K,order", [
+    (wl.OP_AG_GEMM, 4, 1024, 2568, 200, api.ORDER_RANK_MAJOR),      # 512x256 and 256x256 tiles, ragged N, K tail
+    (wl.OP_AG_GEMM, 4, 1024, 2568, 424, api.ORDER_STEP_MAJOR),
+    (wl.OP_GEMM_RS, 8, 1024, 2568, 88, api.ORDER_RANK_MAJOR),       # K segments with partial stages
+])
+def test_kn_weights_big_and_small_tiles(op, P, m, N, K, order):
+    w = small(op, P, m, N, K, dist=0.05)
+    A, B = wl.make_inputs(w)
+    outs = run_with_kn_weights(w, A, B, order=order)
+    check_all(outs, ops.ag_gemm(A, B) if op == wl.OP_AG_GEMM else ops.gemm_rs(A, B), w.name)
+
+
+def test_kn_weights_give_the_same_bits_as_nk_weights():
+    """The layout changes how the tile is fetched, not what is multiplied: bit-identical outputs."""
+    for op, P, m, N, K in ((wl.OP_AG_GEMM, 4, 1024, 1032, 456), (wl.OP_GEMM_RS, 4, 512, 776, 200), (wl.OP_AG_GEMM, 2, 96, 264, 72)):
+        w = small(op, P, m, N, K, dist=0.05)
+        A, B = wl.make_inputs(w)
+        kn = run_with_kn_weights(w, A, B)
+        nk, status, guards = gu.run_fused(w, A, B)
+        assert status == (api.OK, 0) and guards
+        for x, y in zip(kn, nk):
+            assert (x == y).all()
+
+
+def test_kn_weights_ring_rmw_and_integer_inputs():
+    w = small(wl.OP_GEMM_RS, 4, 512, 520, 344)
+    A, B = wl.make_structured_inputs(w, "index")
+    outs = run_with_kn_weights(w, A, B, rs_variant=api.RS_RING_RMW)
+    refs = ops.gemm_rs(A, B)
+    for r in range(w.P):
+        assert (ops.bf16_bits_to_f64(outs[r]) == refs[r]).all()
+
+
+def test_kn_weights_interdecom():
+    w = small(wl.OP_AG_GEMM, 4, 512, 520, 200)
+    A_bits, B_bits = wl.make_inputs(w)
+    for d in (1, 4):
+        pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, d=d, b_layout=api.B_KN)
+        A = [api.to_device(a) for a in A_bits]
+        B = [api.to_device(np.ascontiguousarray(b.T)) for b in B_bits]
+        outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        ws = api.alloc_workspace(pr, api.WS_DECOMP)
+        api.compass_decomp(pr, A, B, [o.view for o in outs], ws, torch.cuda.current_stream(), torch.cuda.Stream())
+        assert api.compass_read_status(ws) == (api.OK, 0)
+        torch.cuda.synchronize()
+        check_all([o.bits() for o in outs], ops.decomp_ag_gemm(A_bits, B_bits, d), f"{w.name} d={d}")
