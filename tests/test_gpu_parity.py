@@ -488,3 +488,45 @@ def test_kn_weights_interdecom():
         assert api.compass_read_status(ws) == (api.OK, 0)
         torch.cuda.synchronize()
         check_all([o.bits() for o in outs], ops.decomp_ag_gemm(A_bits, B_bits, d), f"{w.name} d={d}")
+
+
+# ---- seeded sweep over random shapes and options ---------------------------------------------------------
+
+def _random_cases(n, seed):
+    """Shapes drawn so that all three kernels, ragged rows and columns, K tails, K segments, both rings,
+    both launch orders, both reduce variants and both weight layouts occur."""
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < n:
+        op = int(rng.integers(0, 2))
+        P = int(rng.choice([1, 2, 3, 4, 5, 8]))
+        rings = int(rng.choice([1, 2]))
+        m = int(rng.choice([8, 40, 128, 136, 256, 264, 512, 520, 768, 1024])) * (1 if rng.random() < 0.7 else 2)
+        if m % rings:
+            continue
+        N = int(rng.choice([8, 64, 200, 256, 264, 512, 776, 1032]))
+        K = int(rng.choice([8, 16, 64, 72, 128, 200, 320, 384, 392, 456, 1024]))
+        if P * m * N * K * P > 6e10:            # keep the FP64 oracle to about a second per case
+            continue
+        cases.append((op, P, m, N, K, rings, int(rng.integers(0, 2)), int(rng.integers(0, 2)), int(rng.integers(0, 2))))
+    return cases
+
+
+@pytest.mark.parametrize("op,P,m,N,K,rings,order,variant,layout", _random_cases(40, seed=20261125))
+def test_random_shapes_and_options(op, P, m, N, K, rings, order, variant, layout):
+    w = small(op, P, m, N, K, seed=P + m + N + K, dist=0.1)
+    A_bits, B_bits = wl.make_inputs(w)
+    rs_variant = api.RS_RING_RMW if (op == wl.OP_GEMM_RS and variant) else api.RS_SEGMENTED_K
+    pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, rings=rings, rs_variant=rs_variant, order=order, b_layout=layout)
+    A = [api.to_device(a) for a in A_bits]
+    B = [api.to_device(np.ascontiguousarray(b.T) if layout == api.B_KN else b) for b in B_bits]
+    outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    ws = api.alloc_workspace(pr)
+    (api.compass_ag_gemm if op == wl.OP_AG_GEMM else api.compass_gemm_rs)(pr, A, B, [o.view for o in outs], ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    assert all(o.guards_intact() for o in outs)
+    refs = ops.ag_gemm(A_bits, B_bits, rings=rings) if op == wl.OP_AG_GEMM else ops.gemm_rs(A_bits, B_bits, rings=rings)
+    for r, (o, ref) in enumerate(zip(outs, refs)):
+        rep = compare.check(o.bits(), ref)
+        limit = np.sqrt(P) * 2.0 ** -9 if rs_variant == api.RS_RING_RMW else compare.RMS_REL_LIMIT
+        assert rep.violations == 0 and rep.rms_rel <= max(limit, compare.RMS_REL_LIMIT), f"rank {r}: {rep}"
