@@ -606,11 +606,33 @@ __device__ __forceinline__ MixedTile decode_mixed(const GemmParams& p, int t) {
   if (t < p.n_big) {
     m.big = 1;
     tb = t;
-  } else {
+  } else if (p.h_last == 2) {
     m.big = 0;
     const int u = t - p.n_big;
     tb = p.n_big + (u >> 1);
     half = u & 1;
+  } else {
+    // A block's last 512-row slot holds at most 256 rows (then the launch has no 512x256 tiles): its second
+    // half does not exist and is not numbered, so that every tile index is a tile and consecutive indices
+    // spread evenly over the pairs.  Per block: full slot rows (2 halves x tiles_n), then the short one.
+    m.big = 0;
+    const int per_block_small = (2 * (p.big_tiles_m - 1) + 1) * p.tiles_n;
+    m.blk = t / per_block_small;
+    int w = t - m.blk * per_block_small;
+    const int full = 2 * (p.big_tiles_m - 1) * p.tiles_n;
+    int mtb;
+    if (w < full) {
+      mtb = w / (2 * p.tiles_n);
+      w -= mtb * 2 * p.tiles_n;
+      m.nt = w >> 1;
+      half = w & 1;
+    } else {
+      mtb = p.big_tiles_m - 1;
+      m.nt = w - full;
+    }
+    m.row0 = mtb * (4 * BM) + half * (2 * BM);
+    m.valid = m.row0 < p.rows_per_block;
+    return m;
   }
   const int per_block = p.big_tiles_m * p.tiles_n;
   m.blk = tb / per_block;
@@ -1187,7 +1209,9 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
     const int total_big = L.n_blocks * p.big_tiles_m * p.tiles_n;
     const bool use_big = L.rows_per_block % (4 * BM) == 0;
     p.n_big = use_big ? (total_big / info->max_pairs) * info->max_pairs : 0;
-    p.total_tiles = p.n_big + 2 * (total_big - p.n_big);
+    p.h_last = (L.rows_per_block - (p.big_tiles_m - 1) * 4 * BM > 2 * BM) ? 2 : 1;
+    p.total_tiles = p.h_last == 2 ? p.n_big + 2 * (total_big - p.n_big)
+                                  : L.n_blocks * (2 * (p.big_tiles_m - 1) + 1) * p.tiles_n;
     p.kb_big = int32_t((L.K + BK - 1) / BK);
     p.tail_big = int32_t((L.K - int64_t(p.kb_big - 1) * BK + UMMA_K - 1) / UMMA_K);
   }

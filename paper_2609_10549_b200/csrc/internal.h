@@ -90,6 +90,7 @@ struct GemmParams {
   // mixed-tile pair kernel: tiles [0, n_big) are 512x256, the rest 256x256 (two per remaining big tile)
   int32_t n_big;
   int32_t big_tiles_m;     // 512-row tiles per block
+  int32_t h_last;          // 256-row halves of a block's last 512-row slot that hold rows: 2, or 1 when at most 256 rows are left
   int32_t kb_big;          // 64-wide k-stages per segment of a big tile
   int32_t tail_big;        // UMMA_K steps in its last stage
   int32_t epilogue;        // EpilogueMode
