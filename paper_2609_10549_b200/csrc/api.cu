@@ -346,9 +346,10 @@ int decomp_ag(const compass_problem* pr, const void* const* A, const void* const
     if ((e = cudaEventRecord(ev[1 + j], s_copy)) != cudaSuccess) return record_cuda_error(e);
     if ((e = cudaStreamWaitEvent(s_comp, ev[1 + j], 0)) != cudaSuccess) return record_cuda_error(e);
     // sub-GEMM j on the gathered rows
+    // rank-major, like the fused launch: a rank's weight shard stays in L2 across its P row slices
     int n = 0;
-    for (int q = 0; q < P; ++q)
-      for (int r = 0; r < P; ++r) {
+    for (int r = 0; r < P; ++r)
+      for (int q = 0; q < P; ++q) {
         BlockDesc& b = L.blocks[n++];
         std::memset(&b, 0, sizeof(b));
         b.a_map = uint8_t(r);
@@ -392,9 +393,10 @@ int decomp_rs(const compass_problem* pr, const void* const* A, const void* const
   cudaError_t e;
   for (int j = 0; j < d; ++j) {
     // sub-GEMM j: every rank's partial rows of slice j of every owner's block
+    // rank-major: rank q's weight shard stays in L2 across the P owners' row slices
     int n = 0;
-    for (int c = 0; c < P; ++c)
-      for (int q = 0; q < P; ++q) {
+    for (int q = 0; q < P; ++q)
+      for (int c = 0; c < P; ++c) {
         BlockDesc& b = L.blocks[n++];
         std::memset(&b, 0, sizeof(b));
         b.a_map = uint8_t(q);
