@@ -193,7 +193,12 @@ int compass_ag_gemm(const compass_problem* problem, const void* const* A, const 
  * COMPASS_ERR_TIMEOUT).  Tiles are issued step-major (all ranks in lockstep).
  * Arguments as compass_ag_gemm; workspace >= compass_workspace_bytes(problem,
  * COMPASS_WS_PUSH).  On return all work is ordered before later work on
- * stream_compute.  stream_copy must differ from stream_compute. */
+ * stream_compute.  stream_copy must differ from stream_compute.  With two
+ * rings the backward ring's copy chain runs on stream_copy and the forward
+ * ring's on a stream of the library's own (one per device, created on first
+ * use): the rings move disjoint partitions, so their chains are independent.
+ * The kernel is launched before the copies are enqueued, so that it does not
+ * wait for the host to issue them. */
 int compass_ag_gemm_push(const compass_problem* problem, const void* const* A, const void* const* B,
                          void* const* C, void* workspace, size_t workspace_bytes,
                          void* stream_compute, void* stream_copy);

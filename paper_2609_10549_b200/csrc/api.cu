@@ -282,6 +282,20 @@ struct EventPool {
   cudaEvent_t all[kMaxDevices][2 * 16 + 2];
   int made[kMaxDevices] = {};
   cudaEvent_t* ev = nullptr;      // the current device's set, valid after ensure()
+  cudaStream_t side_stream[kMaxDevices] = {};   // second copy stream of the push variant, created on first use
+  // A non-blocking stream of the library's own on the current device (under `mu`).
+  int ensure_side_stream(cudaStream_t* out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (dev < 0 || dev >= kMaxDevices) return COMPASS_ERR_UNSUPPORTED;
+    if (side_stream[dev] == nullptr) {
+      e = cudaStreamCreateWithFlags(&side_stream[dev], cudaStreamNonBlocking);
+      if (e != cudaSuccess) return record_cuda_error(e);
+    }
+    *out = side_stream[dev];
+    return COMPASS_OK;
+  }
   int ensure(int n) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -660,12 +674,25 @@ extern "C" int compass_ag_gemm_push(const compass_problem* pr, const void* const
 
   cudaStream_t sc = static_cast<cudaStream_t>(stream_compute), sp = static_cast<cudaStream_t>(stream_copy);
   std::lock_guard<std::mutex> lock(g_events.mu);
-  st = g_events.ensure(2);
+  st = g_events.ensure(3);
   if (st != COMPASS_OK) return st;
+  // The two rings move independent partitions (a partition travels along one ring only), so their copy chains
+  // run on two streams: the caller's copy stream and one of the library's own.  One chain of 2(P-1)P small
+  // copies, each followed by a flag write, would otherwise be what the GEMM waits for.
+  cudaStream_t ring_stream[2] = {sp, sp};
+  if (rings == 2) {
+    st = g_events.ensure_side_stream(&ring_stream[1]);
+    if (st != COMPASS_OK) return st;
+  }
   cudaError_t e;
   // the pushes start after whatever precedes this call on the compute stream (inputs ready, buffers free)
   if ((e = cudaEventRecord(g_events.ev[0], sc)) != cudaSuccess) return record_cuda_error(e);
   if ((e = cudaStreamWaitEvent(sp, g_events.ev[0], 0)) != cudaSuccess) return record_cuda_error(e);
+  if (rings == 2 && (e = cudaStreamWaitEvent(ring_stream[1], g_events.ev[0], 0)) != cudaSuccess) return record_cuda_error(e);
+  // The kernel goes first: its step-0 tiles need nothing, and the host needs a while to enqueue the 2(P-1)P
+  // copies and flag writes that follow (tiles of later steps wait, bounded, for their flags).
+  st = launch_gemm(L, sc);
+  if (st != COMPASS_OK) return st;
   const size_t part_bytes = size_t(h) * size_t(K) * 2;
   for (int step = 1; step < P; ++step)
     for (int ring = 0; ring < rings; ++ring)
@@ -676,16 +703,17 @@ extern "C" int compass_ag_gemm_push(const compass_problem* pr, const void* const
                                  ? static_cast<const uint8_t*>(A[peer]) + size_t(en.row_begin - en.chunk * m) * size_t(K) * 2
                                  : G[peer] + size_t(en.row_begin) * size_t(K) * 2;
         uint8_t* dst = G[rank] + size_t(en.row_begin) * size_t(K) * 2;
-        if ((e = cudaMemcpyAsync(dst, src, part_bytes, cudaMemcpyDeviceToDevice, sp)) != cudaSuccess)
+        cudaStream_t s = ring_stream[ring];
+        if ((e = cudaMemcpyAsync(dst, src, part_bytes, cudaMemcpyDeviceToDevice, s)) != cudaSuccess)
           return record_cuda_error(e);
         uint32_t* flag = flags + size_t(rank) * rings * P + en.part;
-        if (write_value(reinterpret_cast<CUstream>(sp), reinterpret_cast<CUdeviceptr>(flag), token, 0) != CUDA_SUCCESS)
+        if (write_value(reinterpret_cast<CUstream>(s), reinterpret_cast<CUdeviceptr>(flag), token, 0) != CUDA_SUCCESS)
           return record_cuda_error(cudaErrorUnknown);
       }
   if ((e = cudaEventRecord(g_events.ev[1], sp)) != cudaSuccess) return record_cuda_error(e);
-  st = launch_gemm(L, sc);
-  if (st != COMPASS_OK) return st;
+  if (rings == 2 && (e = cudaEventRecord(g_events.ev[2], ring_stream[1])) != cudaSuccess) return record_cuda_error(e);
   if ((e = cudaStreamWaitEvent(sc, g_events.ev[1], 0)) != cudaSuccess) return record_cuda_error(e);
+  if (rings == 2 && (e = cudaStreamWaitEvent(sc, g_events.ev[2], 0)) != cudaSuccess) return record_cuda_error(e);
   return COMPASS_OK;
 }
 
