@@ -181,6 +181,29 @@ def test_config4_gemm_rs_full_size_sampled():
     _sampled_rs(wl.C4_RS)
 
 
+# The two operators of the benchmark step, in the configuration bench.py times, every element of every rank.
+def test_config2_ag_gemm_every_element():
+    w = wl.C2_AG
+    A, B = wl.make_inputs(w)
+    outs, status, guards = gu.run_fused(w, A, B)
+    assert status == (api.OK, 0) and guards
+    for r in range(w.P):                                   # one rank at a time keeps the FP64 reference at 100 MB
+        (ref,) = ops.ag_gemm(A, B, ranks=[r])
+        rep = compare.check(outs[r], ref)
+        assert rep.ok and rep.frac_within_1ulp > 0.999, f"{w.name} rank {r}: {rep}"
+
+
+def test_config3_gemm_rs_every_element():
+    w = wl.C3_RS
+    A, B = wl.make_inputs(w)
+    outs, status, guards = gu.run_fused(w, A, B)
+    assert status == (api.OK, 0) and guards
+    for c in range(w.P):
+        (ref,) = ops.gemm_rs(A, B, chunks=[c])
+        rep = compare.check(outs[c], ref)
+        assert rep.ok and rep.frac_within_1ulp > 0.999, f"{w.name} chunk {c}: {rep}"
+
+
 def test_config5_ag_gemm_full_size_sampled():
     _sampled_ag(wl.C5_AG)
 
