@@ -71,8 +71,8 @@ size_t push_flag_count(const compass_problem* pr) { return size_t(pr->P) * size_
 
 // ---- fused launches: schedule -> blocks -------------------------------------
 
-// AllGather+GEMM: one block per schedule entry, listed step-major, then ring,
-// then rank, so that for every rank the blocks appear in its schedule order.
+// AllGather+GEMM: one block per schedule entry.  Rank-major lists the table's own order; step-major lists
+// step, then rank, then ring.  Either way every rank's blocks appear in its schedule order.
 void plan_ag(const compass_problem* pr, const compass_sched_entry* table, GemmLaunch* L, compass_plan_block* view) {
   const int P = pr->P, rings = pr->rings;
   const int64_t m = pr->M / P;
@@ -88,10 +88,10 @@ void plan_ag(const compass_problem* pr, const compass_sched_entry* table, GemmLa
   const bool rank_major = pr->order == COMPASS_ORDER_RANK_MAJOR;
   const int n_entries = P * P * rings;
   for (int i = 0; i < n_entries; ++i) {
-    // rank-major: the table's own order; step-major: step, then ring, then rank
-    const int rank = rank_major ? i / (P * rings) : i % P;
+    // rank-major: the table's own order; step-major: step, then rank, then ring (a rank's entries of one step adjacent)
+    const int rank = rank_major ? i / (P * rings) : (i / rings) % P;
     const int step = rank_major ? (i / rings) % P : i / (rings * P);
-    const int ring = rank_major ? i % rings : (i / P) % rings;
+    const int ring = i % rings;
     const compass_sched_entry& e = table[(size_t(rank) * P + step) * rings + ring];
     BlockDesc& b = L->blocks[n];
     std::memset(&b, 0, sizeof(b));
@@ -173,8 +173,8 @@ void plan_rs_ring(const compass_problem* pr, const compass_sched_entry* table, G
   L->last_step = P - 1;
   int n = 0;
   for (int step = 0; step < P; ++step)
-    for (int ring = 0; ring < rings; ++ring)
-      for (int rank = 0; rank < P; ++rank) {
+    for (int rank = 0; rank < P; ++rank)        // a rank's entries of one step are adjacent: they share its weight shard in L2
+      for (int ring = 0; ring < rings; ++ring) {
         const compass_sched_entry& e = table[(size_t(rank) * P + step) * rings + ring];
         BlockDesc& b = L->blocks[n];
         std::memset(&b, 0, sizeof(b));
@@ -651,8 +651,8 @@ extern "C" int compass_ag_gemm_push(const compass_problem* pr, const void* const
   }
   int n = 0;
   for (int step = 0; step < P; ++step)
-    for (int ring = 0; ring < rings; ++ring)
-      for (int rank = 0; rank < P; ++rank) {
+    for (int rank = 0; rank < P; ++rank)        // a rank's entries of one step are adjacent: they share its weight shard in L2
+      for (int ring = 0; ring < rings; ++ring) {
         const compass_sched_entry& e = table[(size_t(rank) * P + step) * rings + ring];
         BlockDesc& b = L.blocks[n++];
         b = BlockDesc{};
