@@ -685,6 +685,13 @@ extern "C" int compass_ag_gemm_push(const compass_problem* pr, const void* const
     if (st != COMPASS_OK) return st;
   }
   cudaError_t e;
+  // Inside a stream capture the token is frozen into the graph, so a replay would find the flags of the
+  // previous replay already up: the captured work then starts by clearing them.
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  if ((e = cudaStreamIsCapturing(sc, &capturing)) != cudaSuccess) return record_cuda_error(e);
+  if (capturing == cudaStreamCaptureStatusActive &&
+      (e = cudaMemsetAsync(flags, 0, push_flag_count(pr) * sizeof(uint32_t), sc)) != cudaSuccess)
+    return record_cuda_error(e);
   // the pushes start after whatever precedes this call on the compute stream (inputs ready, buffers free)
   if ((e = cudaEventRecord(g_events.ev[0], sc)) != cudaSuccess) return record_cuda_error(e);
   if ((e = cudaStreamWaitEvent(sp, g_events.ev[0], 0)) != cudaSuccess) return record_cuda_error(e);

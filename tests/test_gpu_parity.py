@@ -553,3 +553,68 @@ def test_random_shapes_and_options(op, P, m, N, K, rings, order, variant, layout
         rep = compare.check(o.bits(), ref)
         limit = np.sqrt(P) * 2.0 ** -9 if rs_variant == api.RS_RING_RMW else compare.RMS_REL_LIMIT
         assert rep.violations == 0 and rep.rms_rel <= max(limit, compare.RMS_REL_LIMIT), f"rank {r}: {rep}"
+
+
+# ---- CUDA graphs -------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("which", ["fused_ag", "fused_rs_rmw", "decomp", "push", "mlp"])
+def test_entry_points_capture_into_cuda_graphs(which):
+    """Every launch path can be captured into a CUDA graph; a replay computes on the CURRENT contents of the
+    input buffers (checked by changing them in place between replays) and gives the bits of the eager call."""
+    w = small(wl.OP_AG_GEMM if which != "fused_rs_rmw" else wl.OP_GEMM_RS, 4, 512, 520, 200, dist=0.05)
+    side = torch.cuda.Stream()
+    A_bits, B_bits = wl.make_inputs(w)
+    A = [api.to_device(a) for a in A_bits]
+    B = [api.to_device(b) for b in B_bits]
+    if which == "mlp":
+        mw = wl.MlpWorkload("graph-mlp", P=4, M=2048, hidden=200, ffn=528, activation=wl.ACT_SWIGLU, seed=2)
+        X_bits, W0_bits, W1_bits = wl.make_mlp_inputs(mw)
+        A = [api.to_device(a) for a in X_bits]
+        W0, W1 = [api.to_device(a) for a in W0_bits], [api.to_device(a) for a in W1_bits]
+        H = [torch.zeros((mw.M, mw.hc), dtype=torch.bfloat16, device="cuda") for _ in range(4)]
+        outs = [torch.zeros((mw.m, mw.hidden), dtype=torch.bfloat16, device="cuda") for _ in range(4)]
+        mp = api.make_mlp(4, mw.M, mw.hidden, mw.ffn, activation=api.ACT_SWIGLU)
+        ws = api.alloc_mlp_workspace(mp)
+        call = lambda: api.compass_mlp_block(mp, A, W0, H, W1, outs, ws, torch.cuda.current_stream())
+    else:
+        outs = [torch.zeros(w.out_shape, dtype=torch.bfloat16, device="cuda") for _ in range(w.P)]
+        if which == "fused_ag":
+            pr = api.make_problem(w.op, w.P, w.M, w.N, w.K)
+            ws = api.alloc_workspace(pr)
+            call = lambda: api.compass_ag_gemm(pr, A, B, outs, ws, torch.cuda.current_stream())
+        elif which == "fused_rs_rmw":
+            pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, rs_variant=api.RS_RING_RMW)
+            ws = api.alloc_workspace(pr)
+            call = lambda: api.compass_gemm_rs(pr, A, B, outs, ws, torch.cuda.current_stream())
+        elif which == "decomp":
+            pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, d=4)
+            ws = api.alloc_workspace(pr, api.WS_DECOMP)
+            call = lambda: api.compass_decomp(pr, A, B, outs, ws, torch.cuda.current_stream(), side)
+        else:
+            pr = api.make_problem(w.op, w.P, w.M, w.N, w.K)
+            ws = api.alloc_workspace(pr, api.WS_PUSH)
+            call = lambda: api.compass_ag_gemm_push(pr, A, B, outs, ws, torch.cuda.current_stream(), side)
+
+    def eager_bits():
+        call()
+        torch.cuda.synchronize()
+        return [o.view(torch.int16).clone() for o in outs]
+
+    first = eager_bits()                                    # also the warm-up the first launch on a device needs
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        call()
+    for trial in range(3):
+        if trial:                                            # new input values in the same buffers
+            for t in A:
+                t.mul_(-0.5 if trial == 1 else 1.25)
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        replayed = [o.view(torch.int16).clone() for o in outs]
+        assert api.compass_read_status(ws) == (api.OK, 0)
+        want = first if trial == 0 else eager_bits()
+        for got, ref in zip(replayed, want):
+            assert bool((got == ref).all()), f"{which}: replay {trial} differs from the eager call"
+        assert any(bool((o != 0).any()) for o in replayed)
