@@ -29,10 +29,11 @@
  * bounded: a wait that gives up records COMPASS_ERR_TIMEOUT in the status
  * block at the start of the workspace (see compass_read_status).
  *
- * CUDA graphs.  Every entry point that launches device work only enqueues
- * kernels, copies, stream memory operations and event record/wait pairs that
- * fork from and join back into the compute stream, so it can be called while
- * that stream is being captured; a replay works on the current contents of
+ * CUDA graphs.  compass_ag_gemm, compass_gemm_rs, compass_decomp,
+ * compass_ag_gemm_push and compass_mlp_block only enqueue kernels, copies,
+ * stream memory operations and event record/wait pairs that fork from and
+ * join back into the compute stream, so they can be called while that stream
+ * is being captured; a replay works on the current contents of
  * the buffers whose addresses were captured.  The first call on a device
  * should come before any capture (it sets kernel attributes and creates the
  * library's events).
