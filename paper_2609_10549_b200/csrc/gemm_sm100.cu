@@ -21,6 +21,12 @@
 //   gemm_kernel<true>  clusters of two CTAs, 256x256 tiles; carries the ring
 //                      read-modify-write epilogue.
 //   gemm_kernel<false> one CTA per 128x256 tile; row fragments below 256 rows.
+// Each has a second instantiation whose plain-store epilogue applies an
+// activation (GELU-tanh, or SwiGLU on interleaved gate/up columns) to the FP32
+// accumulator: the first GEMM of the MLP block (Section II-A).  All of them
+// take the weight tiles either K-contiguous ([N][K]) or N-contiguous ([K][N],
+// MN-major tcgen05 operand), and CTA 0 of every launch records its SM cycles
+// and nanoseconds in the status block.
 // In the pair kernels each CTA loads its own rows of A and its half of the B
 // rows; the leader CTA issues tcgen05.mma.cta_group::2, which reads both CTAs'
 // shared memory, and each CTA's tensor memory receives its rows of the
