@@ -440,7 +440,7 @@ def interdecom_report(torch, api, hbm_gbs):
                         "RS": {f: getattr(cal_rs, f) for f in fields},
                         "shapes": "three shapes per pattern, none of them predicted below"},
         "config4": [predict_and_measure(wl.C4_AG, cal_ag, True), predict_and_measure(wl.C4_RS, cal_rs, True)],
-        "config5": [predict_and_measure(wl.C5_AG, cal_ag, False), predict_and_measure(wl.C5_RS, cal_rs, False)],
+        "config5": [predict_and_measure(wl.C5_AG, cal_ag, True), predict_and_measure(wl.C5_RS, cal_rs, True)],
         "paper_context": "paper (8x RTX A6000, hybrid NVLink-PCIe): IntraFusion 1.5-2.5x over sequential, InterDecom up to "
                          "1.3x over fixed d=4, 1.42x end to end; interconnect gains, not reproducible on one GPU",
     }

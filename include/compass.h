@@ -177,8 +177,9 @@ int compass_schedule(int op, int P, int rings, int64_t M,
  * ONE kernel launch computes C_r for all ranks.  A tile of C_r that belongs
  * to partition p of rank r's schedule reads its A rows directly from the
  * shard of the rank that owns p (the gather is done by address, there is no
- * gather buffer) and is issued in schedule order: step-major; inside a step
- * ranks are interleaved per ring.
+ * gather buffer) and is issued in that rank's schedule order; the P ranks'
+ * sequences are merged rank-major by default, step-major on request
+ * (problem->order).
  *   A: P device pointers, A[r] = [M/P x K];  B: P device pointers [N x K];
  *   C: P device pointers [M x N] (every element is written).
  *   workspace: >= compass_workspace_bytes(problem, COMPASS_WS_FUSED) bytes of
@@ -207,7 +208,13 @@ int compass_ag_gemm(const compass_problem* problem, const void* const* A, const 
  * ring's on a stream of the library's own (one per device, created on first
  * use): the rings move disjoint partitions, so their chains are independent.
  * The kernel is launched before the copies are enqueued, so that it does not
- * wait for the host to issue them. */
+ * wait for the host to issue them.
+ * Precondition: the kernel's tiles wait for flags while holding their SMs, and
+ * its grid is sized for an otherwise idle GPU.  Run nothing else on the GPU's
+ * SMs for the duration of the call (another kernel of this process that
+ * occupies SMs can keep a tile that others wait for from starting; the waits
+ * then run into the limit).  Read compass_read_status after the call: on
+ * COMPASS_ERR_TIMEOUT the output is incomplete. */
 int compass_ag_gemm_push(const compass_problem* problem, const void* const* A, const void* const* B,
                          void* const* C, void* workspace, size_t workspace_bytes,
                          void* stream_compute, void* stream_copy);
@@ -217,7 +224,15 @@ int compass_ag_gemm_push(const compass_problem* problem, const void* const* A, c
  * ring g) the contributions are added in the order in which the running sum
  * would travel the ring, ending with the owner c.
  *   A: P device pointers [M x K];  B: P device pointers [N x K];
- *   Out: P device pointers [M/P x N] (every element is written). */
+ *   Out: P device pointers [M/P x N] (every element is written).
+ * Precondition of COMPASS_RS_RING_RMW: contributor s of an output tile waits,
+ * holding its SM, for contributor s-1, which is earlier in the launch; that
+ * is deadlock-free because all CTAs of the launch are resident at once, and
+ * the grid is sized for an otherwise idle GPU.  Run nothing else on the GPU's
+ * SMs for the duration of the call, and read compass_read_status after it: on
+ * COMPASS_ERR_TIMEOUT the output holds partial sums and the tile counters are
+ * dirty (re-initialise the workspace).  The segmented-K variant has no such
+ * waits. */
 int compass_gemm_rs(const compass_problem* problem, const void* const* A, const void* const* B,
                     void* const* Out, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
@@ -239,12 +254,20 @@ int compass_decomp(const compass_problem* problem, const void* const* A, const v
                    void* const* out, void* workspace, size_t workspace_bytes,
                    void* stream_compute, void* stream_copy);
 
-/* ---- strategy selector (Algorithm 1) -------------------------------------
- * Phase 1: T_comp, T_comm, lambda from the calibrated linear models; phase 2:
- * d* by Eq. 4-5 (restricted to degrees that divide M/P); phase 3: T_decomp
- * (Eq. 2) against T_fusion (Eq. 7-8); IntraFusion only if strictly faster.
- * Host arithmetic only. */
+/* ---- strategy selector (Algorithm 1, Eq. 2-8) ------------------------------
+ * T_comp, T_comm and lambda come from the calibrated linear models; the
+ * decomposition degree d* from Eq. 4-5 (restricted to degrees that divide
+ * M/P); the answer is the strategy with the smaller predicted time, T_decomp
+ * (Eq. 2 at d*) or T_fusion (Eq. 7-8), IntraFusion only if strictly faster.
+ * Host arithmetic only.
+ * compass_select evaluates Eq. 5 with min(lambda, 1/lambda) in place of the
+ * printed 1/lambda -- a deliberate departure: that is the stationary point of
+ * Eq. 2 in both regimes, and it coincides with the printed form whenever
+ * T_comp >= T_comm (see compass_model_optimal_degree).  compass_select_ex with
+ * eq5_as_printed != 0 runs the selector on Eq. 5 exactly as printed. */
 int compass_select(const compass_problem* problem, const compass_calib* calib, compass_choice* out);
+int compass_select_ex(const compass_problem* problem, const compass_calib* calib, int eq5_as_printed,
+                      compass_choice* out);
 
 /* ---- the tensor-parallel MLP block (Section II-A, the two-layer MLP figure) --
  * AllGather -> GEMM0 (W0 column-parallel) -> GEMM1 (W1 row-parallel) ->
@@ -363,20 +386,48 @@ int compass_fused_host(const compass_problem* problem, const void* const* A_host
  * size is refused with COMPASS_ERR_SCRATCH_LIMIT.  The call allocates nothing:
  * no cudaMalloc, no cudaFree, no allocating library routine.
  * The first call on a device looks up the array's device address (once per
- * device, with that device current); make that first call before any stream
- * capture begins.  All calls on a GPU share the array, which keeps what the
+ * device, with that device current; if the CUDA runtime loads modules lazily,
+ * that is also when the driver reserves the array's memory on that GPU); make
+ * that first call before any stream capture begins.  All calls on a GPU share the array, which keeps what the
  * previous call left in it (the status block is cleared at the start of every
  * call; the partials are overwritten before they are read): calls ordered on
  * one stream are fine, calls that overlap on the GPU race and give undefined
- * results.  A device-side wait that gives up is recorded inside the array and
- * cannot be read back through this entry point. */
+ * results.  A device-side wait that gives up is recorded inside the array:
+ * read it with compass_noalloc_read_status before the next no-allocation call
+ * on that GPU (which clears it). */
 int compass_gemm_rs_sequential_noalloc(const compass_problem* problem, const void* const* A, const void* const* B,
                                        void* const* Out, void* cuda_stream);
+/* Companion of the entry point above (the paper has no counterpart): such a
+ * caller never sees a workspace, so compass_read_status has nothing to read.
+ * This call synchronises cuda_stream and returns the device-side status that
+ * the last compass_gemm_rs_sequential_noalloc on the current device left in
+ * the built-in array (COMPASS_OK or COMPASS_ERR_TIMEOUT; *detail, which may be
+ * NULL, tells which wait gave up).  It allocates nothing either.  After
+ * COMPASS_ERR_TIMEOUT the output rows of that call are incomplete.  Call it
+ * before the next no-allocation call on that GPU, which clears the record. */
+int compass_noalloc_read_status(void* cuda_stream, int* detail);
 
 /* Bound, in microseconds, of every device-side wait of later launches (default
  * 2,000,000).  A wait that exceeds it makes the kernel record
  * COMPASS_ERR_TIMEOUT and return instead of spinning.  0 restores the default. */
 int compass_set_wait_limit_us(uint32_t microseconds);
+/* The library keeps the TMA tensor maps it encodes in a small per-thread
+ * table keyed by (base pointer, rows, row length, box): repeated calls on the
+ * same buffers skip the driver's encoding call (about a microsecond per map,
+ * 3P maps per fused launch).  A map describes addresses and shapes, not
+ * contents, so the table never needs invalidating; a changed pointer or shape
+ * is a new key.  This call reports, over all threads since the library was
+ * loaded, how many map requests were served from the table and how many were
+ * encoded (host pointers, both required).  Diagnostics only. */
+int compass_tensor_map_cache_stats(uint64_t* hits, uint64_t* misses);
+/* Failure injection on the host, for tests of the bounded waits (the paper has
+ * no counterpart): the next `count` readiness-flag writes of
+ * compass_ag_gemm_push are left out -- the partition is copied but never
+ * announced, as if a peer's message had been lost -- so the tile that needs it
+ * gives up after the wait limit and the call's status block reads
+ * COMPASS_ERR_TIMEOUT with detail 7 (the readiness-flag wait).  No GPU fault is
+ * involved; the context stays usable.  0 switches the injection off. */
+int compass_test_drop_flag_writes(int count);
 const char* compass_status_string(int status);
 int compass_last_cuda_error(void);
 /* Number of kernels this library has launched since it was loaded. */

@@ -181,14 +181,14 @@ class Choice:
     t_star: float
 
 
-def select(op: int, P: int, M: int, N: int, K: int, calib: Calib) -> Choice:
-    """Algorithm 1."""
+def select(op: int, P: int, M: int, N: int, K: int, calib: Calib, as_printed: bool = False) -> Choice:
+    """Algorithm 1.  ``as_printed`` evaluates Eq. 5 literally (1/lambda) inside it."""
     # Phase 1: base metrics
     t_comp = calib.comp_a + calib.comp_b * workload_flops(P, M, N, K)
     t_comm = calib.comm_a + calib.comm_b * workload_comm_bytes(op, P, M, N, K)
     lam = t_comp / t_comm if t_comm > 0 else math.inf
     # Phase 2: parameters and degree
-    d_star = optimal_degree(t_comp, t_comm, calib.alpha_decomp, calib.beta_decomp, max_degree(M, P))
+    d_star = optimal_degree(t_comp, t_comm, calib.alpha_decomp, calib.beta_decomp, max_degree(M, P), as_printed)
     # Phase 3: prediction and selection
     t_decomp = decomp_time(t_comp, t_comm, calib.alpha_decomp, calib.beta_decomp, d_star)
     t_fusion = fusion_time(t_comp, t_comm, P, calib.alpha_fusion, calib.beta_fusion,

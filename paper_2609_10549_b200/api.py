@@ -38,7 +38,7 @@ EXPORTS = (
     "compass_read_status", "compass_launch_plan", "compass_fused_host", "compass_status_string",
     "compass_last_cuda_error", "compass_kernel_launch_count", "compass_gemm_rs_sequential_noalloc",
     "compass_set_wait_limit_us", "compass_calib_fit_line", "compass_ag_gemm_push", "compass_read_kernel_clock",
-    "compass_mlp_workspace_bytes", "compass_mlp_block",
+    "compass_mlp_workspace_bytes", "compass_mlp_block", "compass_noalloc_read_status", "compass_select_ex", "compass_test_drop_flag_writes", "compass_tensor_map_cache_stats",
 )
 
 
@@ -99,6 +99,7 @@ def lib() -> C.CDLL:
         L.compass_mlp_workspace_bytes.argtypes = [C.POINTER(Mlp), C.POINTER(C.c_size_t)]
         L.compass_mlp_block.argtypes = [C.POINTER(Mlp), pp, pp, pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p]
         L.compass_select.argtypes = [C.POINTER(Problem), C.POINTER(Calib), C.POINTER(Choice)]
+        L.compass_select_ex.argtypes = [C.POINTER(Problem), C.POINTER(Calib), C.c_int, C.POINTER(Choice)]
         L.compass_model_decomp_time.argtypes = [C.c_double] * 4 + [C.c_int, C.POINTER(C.c_double)]
         L.compass_model_optimal_degree.argtypes = [C.c_double] * 4 + [C.c_int, C.c_int, C.POINTER(C.c_int),
                                                                        C.POINTER(C.c_double)]
@@ -116,7 +117,10 @@ def lib() -> C.CDLL:
         L.compass_fused_host.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t),
                                          C.c_void_p, C.c_size_t, C.c_void_p]
         L.compass_gemm_rs_sequential_noalloc.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p]
+        L.compass_noalloc_read_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
         L.compass_set_wait_limit_us.argtypes = [C.c_uint32]
+        L.compass_test_drop_flag_writes.argtypes = [C.c_int]
+        L.compass_tensor_map_cache_stats.argtypes = [C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
         L.compass_status_string.argtypes = [C.c_int]
         L.compass_status_string.restype = C.c_char_p
         L.compass_last_cuda_error.restype = C.c_int
@@ -135,6 +139,17 @@ def last_cuda_error() -> int:
 
 def compass_set_wait_limit_us(microseconds: int) -> None:
     _check(lib().compass_set_wait_limit_us(int(microseconds)), "compass_set_wait_limit_us")
+
+
+def compass_test_drop_flag_writes(count: int) -> None:
+    _check(lib().compass_test_drop_flag_writes(int(count)), "compass_test_drop_flag_writes")
+
+
+def tensor_map_cache_stats():
+    """(hits, misses) of the library's table of encoded TMA tensor maps since it was loaded."""
+    hits, misses = C.c_uint64(0), C.c_uint64(0)
+    _check(lib().compass_tensor_map_cache_stats(C.byref(hits), C.byref(misses)), "compass_tensor_map_cache_stats")
+    return int(hits.value), int(misses.value)
 
 
 def kernel_launch_count() -> int:
@@ -164,9 +179,12 @@ def compass_schedule(op: int, P: int, rings: int, M: int) -> np.ndarray:
     return np.frombuffer(buf, dtype=np.int32).reshape(n.value, 8).copy()
 
 
-def compass_select(problem: Problem, calib: Calib) -> Choice:
+def compass_select(problem: Problem, calib: Calib, eq5_as_printed: bool = False) -> Choice:
     out = Choice()
-    _check(lib().compass_select(C.byref(problem), C.byref(calib), C.byref(out)), "compass_select")
+    if eq5_as_printed:
+        _check(lib().compass_select_ex(C.byref(problem), C.byref(calib), 1, C.byref(out)), "compass_select_ex")
+    else:
+        _check(lib().compass_select(C.byref(problem), C.byref(calib), C.byref(out)), "compass_select")
     return out
 
 
@@ -334,6 +352,14 @@ def compass_gemm_rs_sequential_noalloc(problem: Problem, A: Sequence, B: Sequenc
     Refuses problems needing more than NOALLOC_SCRATCH_BYTES."""
     _check(lib().compass_gemm_rs_sequential_noalloc(C.byref(problem), _ptr_array(A), _ptr_array(B), _ptr_array(Out),
                                                     _stream_handle(stream)), "compass_gemm_rs_sequential_noalloc")
+
+
+def compass_noalloc_read_status(stream=None):
+    """(status, detail) the last compass_gemm_rs_sequential_noalloc on the current device left in the
+    built-in array; synchronises the stream, allocates nothing."""
+    detail = C.c_int(0)
+    st = lib().compass_noalloc_read_status(_stream_handle(stream), C.byref(detail))
+    return int(st), int(detail.value)
 
 
 def compass_fused_host_bytes(problem: Problem) -> int:

@@ -13,6 +13,7 @@ namespace {
 std::atomic<int> g_last_cuda_error{0};
 std::atomic<uint64_t> g_kernel_launches{0};
 std::atomic<uint32_t> g_wait_limit_us{0};
+std::atomic<int> g_drop_flag_writes{0};      // host-side failure injection: readiness-flag writes still to be left out
 
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -86,6 +87,10 @@ void plan_ag(const compass_problem* pr, const compass_sched_entry* table, GemmLa
   L->epilogue = EPI_STORE;
   int n = 0;
   const bool rank_major = pr->order == COMPASS_ORDER_RANK_MAJOR;
+  // Runs of consecutive blocks that read the same weight shard: rank-major, all of a rank's entries; step-major, the
+  // ring entries of one step of a rank.  Partitions below 256 rows are tiled in groups out of such a run (with two
+  // rings: the two entries of one step, one CTA of a pair on each).
+  L->share_run = rank_major ? rings * P : rings;
   const int n_entries = P * P * rings;
   for (int i = 0; i < n_entries; ++i) {
     // rank-major: the table's own order; step-major: step, then rank, then ring (a rank's entries of one step adjacent)
@@ -128,6 +133,7 @@ void plan_rs_segmented(const compass_problem* pr, const compass_sched_entry* tab
   L->ldo = pr->N;
   L->n_seg = P;
   L->rows_per_block = int(h);
+  L->share_run = 1;      // every partition walks the ranks' K slices in its own ring order: no two blocks share a B tile
   L->epilogue = EPI_STORE;
   const int n_parts = rings * P;
   for (int part = 0; part < n_parts; ++part) {
@@ -169,6 +175,7 @@ void plan_rs_ring(const compass_problem* pr, const compass_sched_entry* table, G
   L->ldo = pr->N;
   L->n_seg = 1;
   L->rows_per_block = int(m / rings);
+  L->share_run = rings;  // a rank's two ring entries of one step are adjacent and multiply by the same B_rank
   L->epilogue = EPI_RING_RMW;
   L->last_step = P - 1;
   int n = 0;
@@ -329,6 +336,7 @@ int decomp_ag(const compass_problem* pr, const void* const* A, const void* const
   L.ldo = pr->N;
   L.n_seg = 1;
   L.rows_per_block = int(sl);
+  L.share_run = P;       // rank r's P row slices are adjacent and multiply by B_r
   L.epilogue = EPI_STORE;
   L.status = reinterpret_cast<StatusBlock*>(ws);
   L.tile_counters = nullptr;
@@ -396,6 +404,7 @@ int decomp_rs(const compass_problem* pr, const void* const* A, const void* const
   L.ldo = pr->N;
   L.n_seg = 1;
   L.rows_per_block = int(sl);
+  L.share_run = P;       // rank q's P row slices (one per owner) are adjacent and multiply by B_q
   L.epilogue = EPI_STORE;
   L.status = reinterpret_cast<StatusBlock*>(ws);
   L.tile_counters = nullptr;
@@ -528,16 +537,15 @@ extern "C" int compass_gemm_rs(const compass_problem* pr, const void* const* A, 
 // cuStreamWriteValue32: a stream-ordered 32-bit store executed by the front end (no SM, no copy engine).
 typedef CUresult (*StreamWriteValue32Fn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
 static StreamWriteValue32Fn stream_write_fn() {
-  static StreamWriteValue32Fn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  // looked up once; the initialisation of a function-local static is thread-safe
+  static const StreamWriteValue32Fn fn = [] {
     void* ptr = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
         q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<StreamWriteValue32Fn>(ptr);
-  }
+      return reinterpret_cast<StreamWriteValue32Fn>(ptr);
+    return static_cast<StreamWriteValue32Fn>(nullptr);
+  }();
   return fn;
 }
 
@@ -637,6 +645,7 @@ extern "C" int compass_ag_gemm_push(const compass_problem* pr, const void* const
   L.ldo = pr->N;
   L.n_seg = 1;
   L.rows_per_block = int(h);
+  L.share_run = rings;
   L.epilogue = EPI_STORE;
   L.status = reinterpret_cast<StatusBlock*>(ws);
   L.flags = flags;
@@ -714,6 +723,8 @@ extern "C" int compass_ag_gemm_push(const compass_problem* pr, const void* const
         if ((e = cudaMemcpyAsync(dst, src, part_bytes, cudaMemcpyDeviceToDevice, s)) != cudaSuccess)
           return record_cuda_error(e);
         uint32_t* flag = flags + size_t(rank) * rings * P + en.part;
+        // failure injection for tests of the bounded flag wait: the copy is made, its flag is never raised
+        if (g_drop_flag_writes.load(std::memory_order_relaxed) > 0 && g_drop_flag_writes.fetch_sub(1) > 0) continue;
         if (write_value(reinterpret_cast<CUstream>(s), reinterpret_cast<CUdeviceptr>(flag), token, 0) != CUDA_SUCCESS)
           return record_cuda_error(cudaErrorUnknown);
       }
@@ -801,6 +812,16 @@ extern "C" const char* compass_status_string(int status) {
 
 extern "C" int compass_set_wait_limit_us(uint32_t microseconds) {
   g_wait_limit_us.store(microseconds, std::memory_order_relaxed);
+  return COMPASS_OK;
+}
+extern "C" int compass_tensor_map_cache_stats(uint64_t* hits, uint64_t* misses) {
+  if (hits == nullptr || misses == nullptr) return COMPASS_ERR_INVALID_ARG;
+  tensor_map_cache_stats(hits, misses);
+  return COMPASS_OK;
+}
+extern "C" int compass_test_drop_flag_writes(int count) {
+  if (count < 0) return COMPASS_ERR_INVALID_ARG;
+  g_drop_flag_writes.store(count);
   return COMPASS_OK;
 }
 extern "C" int compass_last_cuda_error(void) { return g_last_cuda_error.load(); }

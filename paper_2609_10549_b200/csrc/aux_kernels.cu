@@ -133,20 +133,17 @@ int launch_reduce_partials(const void* const* partial, int P, void* const* out, 
   p.slice_rows = slice_rows;
   const int64_t total = slice_rows * p.n_vec * P;
   if (total <= 0) return COMPASS_OK;
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return record_cuda_error(e);
-  }
+  int dev = 0, num_sms = 0;      // asked per call: the current device may differ from the last call's
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return record_cuda_error(e);
+  e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return record_cuda_error(e);
   int64_t want = (total + 255) / 256;
   int64_t cap = int64_t(num_sms) * 8;
   int grid = int(want < cap ? want : cap);
   reduce_partials_kernel<<<grid, 256, 0, stream>>>(p);
   count_kernel_launch();
-  cudaError_t e = cudaGetLastError();
+  e = cudaGetLastError();
   if (e != cudaSuccess) return record_cuda_error(e);
   return COMPASS_OK;
 }

@@ -36,6 +36,7 @@
 // warp 1 = tensor-memory allocation + MMA issue (one lane), warps 2..5 =
 // epilogue (warp w reads TMEM lanes 32*(w%4)..+31).  Every wait is bounded and
 // reports COMPASS_ERR_TIMEOUT instead of hanging.
+#include <atomic>
 #include <mutex>
 
 #include "internal.h"
@@ -148,9 +149,11 @@ __device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, Con
 }
 
 // Bounded wait until a tile counter in global memory reaches `target`.
+// (Waits on something another CTA or the host must provide give up after 3/4 of the limit, so that the
+// status names them and not one of the barrier waits queued up behind them in the same CTA.)
 __device__ __forceinline__ bool wait_counter(const int* counter, int target, Control* ctl, const GemmParams& p, int tile) {
   const uint64_t t0 = globaltimer_ns();
-  const uint64_t limit = uint64_t(p.wait_limit_us) * 1000ull;
+  const uint64_t limit = uint64_t(p.wait_limit_us) * 750ull;
   for (uint32_t spins = 0; spins < (1u << 30); ++spins) {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
@@ -171,7 +174,7 @@ __device__ __forceinline__ bool wait_ready_flag(const GemmParams& p, const Block
   if (p.flags == nullptr || b.flag1 == 0) return true;
   const uint32_t* flag = p.flags + (b.flag1 - 1);
   const uint64_t t0 = globaltimer_ns();
-  const uint64_t limit = uint64_t(p.wait_limit_us) * 1000ull;
+  const uint64_t limit = uint64_t(p.wait_limit_us) * 750ull;
   for (uint32_t spins = 0; spins < (1u << 30); ++spins) {
     uint32_t v;
     asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
@@ -201,12 +204,27 @@ __device__ __forceinline__ TileCoord decode_tile(const GemmParams& p, int t) {
   return c;
 }
 
+// A 128-row fragment of a tile: which block it lies in and its first row inside that block.  `vblk` is the
+// virtual block (p.group consecutive blocks, each padded to p.sub_pad rows), `v0` the fragment's first
+// virtual row, a multiple of 128.  Fragments past the last block are mapped beyond that block's rows, where
+// every row is masked.
+struct Frag {
+  int blk, r0;
+};
+__device__ __forceinline__ Frag fragment_of(const GemmParams& p, int vblk, int v0) {
+  if (p.group == 1) return Frag{vblk, v0};
+  int j = v0 / p.sub_pad;
+  if (j >= p.group) j = p.group - 1;
+  return Frag{vblk * p.group + j, v0 - j * p.sub_pad};
+}
+
 // Walks the sequence of k-stages one work unit loads: for every tile of the
 // unit (t, t + n_units, ...), every K segment, every k-stage of the segment.
 template <bool kPair>
 struct StageIter {
   int t, step, cta_rank;
   int seg, kb;
+  int blk;                   // block this CTA's 128 rows of A belong to
   int am, bm, a_row, b_row;
   __device__ StageIter(const GemmParams& p, int unit, int n_units, int rank) : t(unit), step(n_units), cta_rank(rank), seg(0), kb(0) {
     if (valid(p)) enter(p);
@@ -214,11 +232,13 @@ struct StageIter {
   __device__ bool valid(const GemmParams& p) const { return t < p.total_tiles; }
   __device__ void enter(const GemmParams& p) {      // refresh what depends on (t, seg)
     const TileCoord tc = decode_tile(p, t);
-    const BlockDesc& b = p.blocks[tc.blk];
-    a_row = b.a_row0 + tc.mt * Cfg<kPair>::kTileRows + cta_rank * BM;
+    const Frag f = fragment_of(p, tc.blk, tc.mt * Cfg<kPair>::kTileRows + cta_rank * BM);
+    const BlockDesc& b = p.blocks[f.blk];
+    blk = f.blk;
+    a_row = b.a_row0 + f.r0;
     b_row = tc.nt * BN + cta_rank * Cfg<kPair>::kBRows;
-    am = (p.n_seg > 1) ? p.seg_rank[tc.blk][seg] : b.a_map;
-    bm = (p.n_seg > 1) ? am : b.b_map;
+    am = (p.n_seg > 1) ? p.seg_rank[tc.blk][seg] : b.a_map;      // segmented K: blocks are never grouped
+    bm = (p.n_seg > 1) ? am : b.b_map;                           // the blocks of a group share their B tensor
   }
   __device__ void next(const GemmParams& p) {
     if (++kb < p.kb_per_seg) return;
@@ -304,7 +324,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       int ready_t = -1;
       while (ld.valid(p)) {
         if (ld.t != ready_t) {      // first stage of a tile: its A rows may still be on their way
-          if (!wait_ready_flag(p, p.blocks[decode_tile(p, ld.t).blk], ctl, ld.t)) break;
+          if (!wait_ready_flag(p, p.blocks[ld.blk], ctl, ld.t)) break;
           ready_t = ld.t;
         }
         if (!wait_bounded(&ctl->empty[stage], phase ^ 1u, ctl, p, WAIT_SMEM_EMPTY, ld.t)) break;
@@ -448,9 +468,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     }
   } else {
     // ---------------------------------------------------------------- epilogue
-    constexpr int kWarpsPerTile = kPair ? 2 * kEpilogueWarps : kEpilogueWarps;
     const int quarter = warp & 3;               // TMEM lanes this warp may touch
-    const int row_in_tile = int(cta_rank) * BM + quarter * 32 + lane;
     uint32_t it = 0;
     for (int t = unit; t < p.total_tiles; t += n_units, ++it) {
       const uint32_t buf = it & 1u;
@@ -458,8 +476,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       if (!wait_bounded(&ctl->acc_full[buf], acc_phase, ctl, p, WAIT_ACC_FULL, t)) break;
       tc_fence_after_sync();
       const TileCoord tc = decode_tile(p, t);
-      const BlockDesc& b = p.blocks[tc.blk];
-      const int row_in_block = tc.mt * C::kTileRows + row_in_tile;
+      const Frag frag = fragment_of(p, tc.blk, tc.mt * C::kTileRows + int(cta_rank) * BM);   // this CTA's 128 rows
+      const BlockDesc& b = p.blocks[frag.blk];
+      const int row_in_block = frag.r0 + quarter * 32 + lane;
       const bool row_ok = row_in_block < p.rows_per_block;
       const int ncols = min(BN, p.N - tc.nt * BN);
       const int nchunks = (ncols + 31) >> 5;
@@ -471,17 +490,21 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 
       // Ring read-modify-write: contributor `step` of a partition adds its
       // partial tile to the running sum that contributor step-1 left in the
-      // owner's rows.  One counter per output tile counts the epilogue warps
-      // that have finished; contributor s starts when all warps of s-1 have.
-      const bool rmw = p.epilogue == EPI_RING_RMW;
+      // owner's rows.  One counter per 128 x 256 fragment of the output counts
+      // the epilogue warps that have finished; contributor s starts when all
+      // four warps of s-1 have.  (Per fragment, not per tile: the two CTAs of a
+      // pair may be working on different partitions.)
+      const bool rmw = p.epilogue == EPI_RING_RMW && frag.r0 < p.rows_per_block;   // a fragment past the block adds nothing
       const bool add_previous = rmw && b.step > 0;
       int* counter = nullptr;
       if (rmw) {
-        counter = p.tile_counters + (int64_t(b.part) * p.tiles_m + tc.mt) * p.tiles_n + tc.nt;
+        counter = p.tile_counters + (int64_t(b.part) * p.frags_m + frag.r0 / BM) * p.tiles_n + tc.nt;
         if (add_previous) {
           int ready = 1;
-          if (lane == 0) ready = wait_counter(counter, int(b.step) * kWarpsPerTile, ctl, p, t) ? 1 : 0;
+          if (lane == 0) ready = wait_counter(counter, int(b.step) * kEpilogueWarps, ctl, p, t) ? 1 : 0;
           ready = __shfl_sync(0xffffffffu, ready, 0);
+          // lane 0 acquired the counter; the warp barrier orders the other lanes' loads of the running sum behind it
+          __syncwarp();
           if (!ready) break;
         }
       }
@@ -554,7 +577,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         if (lane == 0) {
           const int before = atomicAdd(counter, 1);
           // the last warp of the last contributor leaves the counter at zero for the next call
-          if (int(b.step) == p.last_step && before == (p.last_step + 1) * kWarpsPerTile - 1) atomicExch(counter, 0);
+          if (int(b.step) == p.last_step && before == (p.last_step + 1) * kEpilogueWarps - 1) atomicExch(counter, 0);
         }
       }
     }
@@ -601,8 +624,8 @@ constexpr size_t kMixedSmemBytes =
 
 struct MixedTile {
   int big;        // 1 = 512x256, 0 = 256x256
-  int blk, nt;
-  int row0;       // first row of the pair's tile inside the block
+  int blk, nt;    // virtual block (p.group blocks), n-tile
+  int row0;       // first row of the pair's tile inside the virtual block
   int valid;
 };
 __device__ __forceinline__ MixedTile decode_mixed(const GemmParams& p, int t) {
@@ -637,7 +660,7 @@ __device__ __forceinline__ MixedTile decode_mixed(const GemmParams& p, int t) {
       m.nt = w - full;
     }
     m.row0 = mtb * (4 * BM) + half * (2 * BM);
-    m.valid = m.row0 < p.rows_per_block;
+    m.valid = m.row0 < p.vrows;
     return m;
   }
   const int per_block = p.big_tiles_m * p.tiles_n;
@@ -646,7 +669,7 @@ __device__ __forceinline__ MixedTile decode_mixed(const GemmParams& p, int t) {
   const int mtb = w / p.tiles_n;
   m.nt = w - mtb * p.tiles_n;
   m.row0 = mtb * (4 * BM) + half * (2 * BM);
-  m.valid = m.row0 < p.rows_per_block;
+  m.valid = m.row0 < p.vrows;
   return m;
 }
 
@@ -655,7 +678,8 @@ struct MixedIter {
   int t, step, cta_rank;
   int seg, kb, n_kb;
   MixedTile tile;
-  int am, bm, a_row, b_row;
+  int blk0, blk1;            // blocks of this CTA's 128-row fragments (blk1: second fragment of a 512x256 tile)
+  int am, am1, bm, a_row, a_row1, b_row;
   __device__ MixedIter(const GemmParams& p, int unit, int n_units, int rank) : t(unit), step(n_units), cta_rank(rank), seg(0), kb(0) {
     skip_invalid(p);
   }
@@ -671,11 +695,19 @@ struct MixedIter {
     }
   }
   __device__ void enter(const GemmParams& p) {
-    const BlockDesc& b = p.blocks[tile.blk];
-    a_row = b.a_row0 + tile.row0 + cta_rank * (tile.big ? 2 * BM : BM);
+    const int v0 = tile.row0 + cta_rank * (tile.big ? 2 * BM : BM);
+    const Frag f0 = fragment_of(p, tile.blk, v0);
+    const Frag f1 = tile.big ? fragment_of(p, tile.blk, v0 + BM) : f0;
+    const BlockDesc& b0 = p.blocks[f0.blk];
+    const BlockDesc& b1 = p.blocks[f1.blk];
+    blk0 = f0.blk;
+    blk1 = f1.blk;
+    a_row = b0.a_row0 + f0.r0;
+    a_row1 = b1.a_row0 + f1.r0;
     b_row = tile.nt * BN + cta_rank * (BN / 2);
-    am = (p.n_seg > 1) ? p.seg_rank[tile.blk][seg] : b.a_map;
-    bm = (p.n_seg > 1) ? am : b.b_map;
+    am = (p.n_seg > 1) ? p.seg_rank[tile.blk][seg] : b0.a_map;      // segmented K: blocks are never grouped
+    am1 = (p.n_seg > 1) ? am : b1.a_map;
+    bm = (p.n_seg > 1) ? am : b0.b_map;                             // the blocks of a group share their B tensor
     n_kb = tile.big ? p.kb_big : p.kb_per_seg;
   }
   __device__ void next(const GemmParams& p) {
@@ -743,7 +775,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
       int ready_t = -1;
       for (MixedIter it(p, unit, n_units, int(cta_rank)); it.valid(p); it.next(p), ++j) {
         if (it.t != ready_t) {      // first stage of a tile: its A rows may still be on their way
-          if (!wait_ready_flag(p, p.blocks[it.tile.blk], ctl, it.t)) break;
+          if (!wait_ready_flag(p, p.blocks[it.blk0], ctl, it.t)) break;
+          if (it.blk1 != it.blk0 && !wait_ready_flag(p, p.blocks[it.blk1], ctl, it.t)) break;
           ready_t = it.t;
         }
         const int big = it.tile.big;
@@ -772,7 +805,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
         if (big) {
           const int kx = it.kb * BK;
           tma_load_2d_pair_hint(c0, &p.a_maps[it.am], full_addr, kx, it.a_row, pol_a);
-          tma_load_2d_pair_hint(c1, &p.a_maps[it.am], full_addr, kx, it.a_row + BM, pol_a);
+          tma_load_2d_pair_hint(c1, &p.a_maps[it.am1], full_addr, kx, it.a_row1, pol_a);
           load_b(c2, kx);
         } else {
           const int kx = it.kb * 2 * BK;
@@ -954,7 +987,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
     for (int t = unit; ok && t < p.total_tiles; t += n_units) {
       const MixedTile tile = decode_mixed(p, t);
       if (!tile.valid) continue;
-      const BlockDesc& b = p.blocks[tile.blk];
       const int ncols = min(BN, p.N - tile.nt * BN);
       const int nchunks = (ncols + 31) >> 5;
       const int n_acc = tile.big ? 2 : 1;
@@ -966,8 +998,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
           break;
         }
         tc_fence_after_sync();
-        // big: this CTA owns rows [256*rank, +256) of the tile, accumulator a holds its 128-row block a
-        const int row_in_block = tile.row0 + (tile.big ? int(cta_rank) * 2 * BM + a * BM : int(cta_rank) * BM) + quarter * 32 + lane;
+        // big: this CTA owns rows [256*rank, +256) of the tile, accumulator a holds its 128-row fragment a
+        const Frag frag = fragment_of(p, tile.blk, tile.row0 + (tile.big ? int(cta_rank) * 2 * BM + a * BM : int(cta_rank) * BM));
+        const BlockDesc& b = p.blocks[frag.blk];
+        const int row_in_block = frag.r0 + quarter * 32 + lane;
         const bool row_ok = row_in_block < p.rows_per_block;
         // SwiGLU halves the columns: accumulator columns (2j, 2j+1) = (gate, up) give output column j
         const int act = kAct ? p.activation : int(ACT_NONE);
@@ -1063,22 +1097,20 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  // looked up once; the initialisation of a function-local static is thread-safe
+  static const EncodeTiledFn fn = [] {
     void* ptr = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess) {
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-  }
+        q == cudaDriverEntryPointSuccess)
+      return reinterpret_cast<EncodeTiledFn>(ptr);
+    return static_cast<EncodeTiledFn>(nullptr);
+  }();
   return fn;
 }
 
 // K-major BF16 matrix [rows x K]; box = BK columns x box_rows rows, 128-byte swizzle, zero fill outside.
-bool encode_kmajor(CUtensorMap* map, const void* ptr, int64_t rows, int64_t K, int box_rows) {
+bool encode_kmajor_uncached(CUtensorMap* map, const void* ptr, int64_t rows, int64_t K, int box_rows) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {cuuint64_t(K), cuuint64_t(rows)};
@@ -1089,6 +1121,49 @@ bool encode_kmajor(CUtensorMap* map, const void* ptr, int64_t rows, int64_t K, i
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
+}
+
+// Encoded tensor maps are kept per host thread in a small direct-mapped table keyed by everything the
+// encoding depends on (base pointer, rows, row length, box rows): a training loop calls the same operator
+// on the same buffers over and over, and the driver call costs about a microsecond per map (3P maps per
+// fused launch, d times that for InterDecom).  A map describes addresses and shapes, not contents, so an
+// entry never goes stale; a different pointer or shape is a different key and is encoded afresh.
+struct MapCache {
+  static constexpr int kEntries = 256;
+  struct Key {
+    const void* ptr;
+    int64_t rows, cols;
+    int32_t box_rows, valid;
+  };
+  Key key[kEntries] = {};
+  alignas(64) CUtensorMap map[kEntries];
+};
+std::atomic<uint64_t> g_map_hits{0}, g_map_misses{0};
+
+bool encode_kmajor(CUtensorMap* map, const void* ptr, int64_t rows, int64_t K, int box_rows) {
+  static thread_local MapCache cache;
+  uint64_t h = uint64_t(reinterpret_cast<uintptr_t>(ptr)) >> 4;
+  h = (h ^ (h >> 17) ^ (uint64_t(rows) * 0x9E3779B97F4A7C15ull) ^ (uint64_t(K) * 0xC2B2AE3D27D4EB4Full) ^ uint64_t(box_rows)) *
+      0xD6E8FEB86659FD93ull;
+  const int slot = int(h >> 56) & (MapCache::kEntries - 1);
+  MapCache::Key& k = cache.key[slot];
+  if (k.valid && k.ptr == ptr && k.rows == rows && k.cols == K && k.box_rows == box_rows) {
+    *map = cache.map[slot];
+    g_map_hits.fetch_add(1, std::memory_order_relaxed);
+    return true;
+  }
+  if (!encode_kmajor_uncached(&cache.map[slot], ptr, rows, K, box_rows)) {
+    k.valid = 0;
+    return false;
+  }
+  k.ptr = ptr;
+  k.rows = rows;
+  k.cols = K;
+  k.box_rows = box_rows;
+  k.valid = 1;
+  *map = cache.map[slot];
+  g_map_misses.fetch_add(1, std::memory_order_relaxed);
+  return true;
 }
 
 struct DeviceInfo {
@@ -1147,6 +1222,11 @@ int device_info(DeviceInfo** out) {
 
 }  // namespace
 
+void tensor_map_cache_stats(uint64_t* hits, uint64_t* misses) {
+  *hits = g_map_hits.load(std::memory_order_relaxed);
+  *misses = g_map_misses.load(std::memory_order_relaxed);
+}
+
 size_t gemm_smem_bytes() {
   size_t m = smem_bytes<true>() > smem_bytes<false>() ? smem_bytes<true>() : smem_bytes<false>();
   return m > kMixedSmemBytes ? m : kMixedSmemBytes;
@@ -1157,13 +1237,56 @@ int gemm_tile_rows(int mode, int rows_per_block) {
   return pair ? 2 * BM : BM;
 }
 
+namespace {
+
+// How the blocks of a launch are tiled: `group` consecutive blocks (padded to sub_pad rows each) per virtual
+// block, and whether the virtual blocks are cut into 256-row tiles for CTA pairs or 128-row tiles for single CTAs.
+struct Tiling {
+  int group, sub_pad;
+  bool pair;
+};
+Tiling choose_tiling(const GemmLaunch& L) {
+  Tiling t;
+  t.sub_pad = (L.rows_per_block + BM - 1) / BM * BM;
+  t.group = 1;
+  if (L.mode == GEMM_MODE_SINGLE) {
+    t.pair = false;
+  } else if (L.mode == GEMM_MODE_PAIR || t.sub_pad >= 2 * BM) {
+    t.pair = true;
+  } else {
+    // One 128-row fragment per block: a CTA pair takes fragments of `group` consecutive blocks that read the
+    // same B tensor (for the fused operators: the two ring entries of one step of a rank, adjacent in that
+    // rank's schedule order).  Segmented K cannot group: its blocks walk the B tensors in different orders.
+    t.pair = false;
+    if (L.n_seg == 1 && L.share_run >= 2 && L.n_blocks % L.share_run == 0) {
+      for (int g = 2; g <= L.share_run; ++g)
+        if (L.share_run % g == 0) {
+          t.group = g;
+          t.pair = true;
+          break;
+        }
+    }
+  }
+  return t;
+}
+
+}  // namespace
+
 int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   static thread_local GemmParams p;
   // an activation goes with the plain store only (the ring read-modify-write adds partial sums)
   if (L.activation != ACT_NONE && L.epilogue != EPI_STORE) return COMPASS_ERR_INVALID_ARG;
   if (L.activation == ACT_SWIGLU && (L.N % 16 != 0 || L.ldo < L.N / 2)) return COMPASS_ERR_INVALID_ARG;
-  const int tile_rows = gemm_tile_rows(L.mode, L.rows_per_block);
-  const bool pair = tile_rows == 2 * BM;
+  DeviceInfo* info = nullptr;
+  int st = device_info(&info);
+  if (st != COMPASS_OK) return st;
+  Tiling tiling = choose_tiling(L);
+  if (tiling.pair && info->max_pairs <= 0) {   // no room for clusters on this device: single-CTA tiles, no grouping needed
+    tiling.pair = false;
+    tiling.group = 1;
+  }
+  const bool pair = tiling.pair;
+  const int tile_rows = pair ? 2 * BM : BM;
   const int b_box_rows = pair ? BN / 2 : BN;
   for (int i = 0; i < L.n_a; ++i)
     if (!encode_kmajor(&p.a_maps[i], L.a_ptr[i], L.a_map_rows[i] ? L.a_map_rows[i] : L.a_rows, L.K, BM))
@@ -1182,9 +1305,14 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   p.kb_per_seg = int32_t((L.K + stage_k - 1) / stage_k);
   const int64_t k_tail = L.K - int64_t(p.kb_per_seg - 1) * stage_k;
   p.tail_ksteps = int32_t((k_tail + UMMA_K - 1) / UMMA_K);
-  p.tiles_m = (L.rows_per_block + tile_rows - 1) / tile_rows;
+  p.group = tiling.group;
+  p.sub_pad = tiling.sub_pad;
+  p.vrows = tiling.group * tiling.sub_pad;
+  p.frags_m = tiling.sub_pad / BM;
+  const int n_vblocks = L.n_blocks / tiling.group;
+  p.tiles_m = (p.vrows + tile_rows - 1) / tile_rows;
   p.tiles_n = int32_t((L.N + BN - 1) / BN);
-  p.total_tiles = L.n_blocks * p.tiles_m * p.tiles_n;
+  p.total_tiles = n_vblocks * p.tiles_m * p.tiles_n;
   p.epilogue = L.epilogue;
   p.last_step = L.last_step;
   p.wait_limit_us = L.wait_limit_us ? L.wait_limit_us : (default_wait_limit_us() ? default_wait_limit_us() : 2000000u);
@@ -1204,25 +1332,25 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
     for (int b = 0; b < L.n_blocks; ++b)
       for (int s = 0; s < L.n_seg; ++s) p.seg_rank[b][s] = L.seg_rank[b][s];
 
-  DeviceInfo* info = nullptr;
-  int st = device_info(&info);
-  if (st != COMPASS_OK) return st;
   if (p.total_tiles <= 0) return COMPASS_OK;
   // Mixed tiles: 512x256 for as many whole waves of pairs as the launch holds, 256x256 for the rest.
-  const bool mixed = pair && info->max_pairs > 0 && L.epilogue == EPI_STORE && L.mode != GEMM_MODE_PAIR;
+  const bool mixed = pair && L.epilogue == EPI_STORE && L.mode != GEMM_MODE_PAIR;
   if (mixed) {
-    p.big_tiles_m = (L.rows_per_block + 4 * BM - 1) / (4 * BM);
-    const int total_big = L.n_blocks * p.big_tiles_m * p.tiles_n;
-    const bool use_big = L.rows_per_block % (4 * BM) == 0;
+    // rows of a (virtual) block that hold data when it is cut into 256-row halves of 512-row slots
+    const int rows = tiling.group > 1 ? p.vrows : L.rows_per_block;
+    p.big_tiles_m = (rows + 4 * BM - 1) / (4 * BM);
+    const int total_big = n_vblocks * p.big_tiles_m * p.tiles_n;
+    const bool use_big = rows % (4 * BM) == 0;
     p.n_big = use_big ? (total_big / info->max_pairs) * info->max_pairs : 0;
-    p.h_last = (L.rows_per_block - (p.big_tiles_m - 1) * 4 * BM > 2 * BM) ? 2 : 1;
+    p.h_last = (rows - (p.big_tiles_m - 1) * 4 * BM > 2 * BM) ? 2 : 1;
+    p.vrows = rows;
     p.total_tiles = p.h_last == 2 ? p.n_big + 2 * (total_big - p.n_big)
-                                  : L.n_blocks * (2 * (p.big_tiles_m - 1) + 1) * p.tiles_n;
+                                  : n_vblocks * (2 * (p.big_tiles_m - 1) + 1) * p.tiles_n;
     p.kb_big = int32_t((L.K + BK - 1) / BK);
     p.tail_big = int32_t((L.K - int64_t(p.kb_big - 1) * BK + UMMA_K - 1) / UMMA_K);
   }
   cudaError_t e;
-  if (pair && info->max_pairs > 0) {
+  if (pair) {
     const int pairs = p.total_tiles < info->max_pairs ? p.total_tiles : info->max_pairs;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(unsigned(2 * pairs));
@@ -1241,14 +1369,6 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
     else if (L.activation != ACT_NONE) e = cudaLaunchKernelEx(&cfg, gemm_kernel<true, true>, p);
     else e = cudaLaunchKernelEx(&cfg, gemm_kernel<true, false>, p);
   } else {
-    if (pair) {   // no room for clusters on this device: fall back to single-CTA tiles
-      p.tiles_m = (L.rows_per_block + BM - 1) / BM;
-      p.total_tiles = L.n_blocks * p.tiles_m * p.tiles_n;
-      p.kb_per_seg = int32_t((L.K + BK - 1) / BK);
-      p.tail_ksteps = int32_t((L.K - int64_t(p.kb_per_seg - 1) * BK + UMMA_K - 1) / UMMA_K);
-      for (int i = 0; i < L.n_b; ++i)
-        if (!L.b_mn_major && !encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, BN)) return record_cuda_error(cudaErrorUnknown);
-    }
     const int grid = p.total_tiles < info->num_sms ? p.total_tiles : info->num_sms;
     if (L.activation != ACT_NONE) gemm_kernel<false, true><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);
     else gemm_kernel<false, false><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);

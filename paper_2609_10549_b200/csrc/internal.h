@@ -85,7 +85,15 @@ struct GemmParams {
   int32_t n_seg;           // K segments accumulated into one tile (1, or P for segmented-K reduce)
   int32_t kb_per_seg;      // k-stages per segment (last one may be partial)
   int32_t tail_ksteps;     // UMMA_K steps in the last k-stage of a segment
-  int32_t tiles_m, tiles_n;
+  // Blocks of fewer than 256 rows that read the same B tensor are tiled together: `group` consecutive blocks,
+  // each padded to `sub_pad` rows (a multiple of 128), form one virtual block of group * sub_pad rows, so that
+  // every 128-row fragment of a tile lies inside ONE block and a CTA pair can work on two blocks at once.
+  // group = 1 and sub_pad >= rows_per_block for ordinary blocks.
+  int32_t group;
+  int32_t sub_pad;
+  int32_t vrows;           // rows of a virtual block: group * sub_pad
+  int32_t frags_m;         // 128-row fragments per block: ceil(rows_per_block / 128)
+  int32_t tiles_m, tiles_n; // tiles per virtual block
   int32_t total_tiles;
   // mixed-tile pair kernel: tiles [0, n_big) are 512x256, the rest 256x256 (two per remaining big tile)
   int32_t n_big;
@@ -122,6 +130,7 @@ struct GemmLaunch {
   int64_t ldo = 0;
   int n_seg = 1;
   int rows_per_block = 0;
+  int share_run = 1;       // blocks come in aligned runs of this many consecutive blocks that read the same B tensor
   int epilogue = EPI_STORE;
   int mode = GEMM_MODE_AUTO;
   int a_hint = 0;   // ptx::L2Hint of the A loads
@@ -144,6 +153,7 @@ struct GemmLaunch {
 // gemm_sm100.cu
 int launch_gemm(const GemmLaunch& launch, cudaStream_t stream);
 size_t gemm_smem_bytes();
+void tensor_map_cache_stats(uint64_t* hits, uint64_t* misses);
 int gemm_tile_rows(int mode, int rows_per_block);   // rows of one scheduling tile: 256 (CTA pair) or 128
 
 // aux_kernels.cu

@@ -183,31 +183,60 @@ extern "C" int compass_calib_fit_fusion(const double* t_comp, const double* t_co
   return ols(xs, ys, k, alpha_f, beta_f) ? COMPASS_OK : COMPASS_ERR_INVALID_ARG;
 }
 
-extern "C" int compass_select(const compass_problem* pr, const compass_calib* cal, compass_choice* out) {
+namespace {
+
+// What the calibrated linear models say about one workload (f and g of Algorithm 1).
+struct BaseTimes {
+  double t_comp, t_comm, volume;
+};
+BaseTimes base_times(const compass_problem* pr, const compass_calib* cal) {
+  const double P = double(pr->P), M = double(pr->M);
+  const double inner = double(pr->op == COMPASS_OP_AG_GEMM ? pr->K : pr->N);   // width of what the collective moves
+  BaseTimes b;
+  b.volume = M * inner;
+  b.t_comp = cal->comp_a + cal->comp_b * (2.0 * P * M * double(pr->N) * double(pr->K));
+  b.t_comm = cal->comm_a + cal->comm_b * (2.0 * P * b.volume);
+  return b;
+}
+
+struct Prediction {
+  int strategy;
+  double time;
+};
+
+}  // namespace
+
+// Algorithm 1 with Eq. 2-8: every strategy gets a predicted time, the fastest wins.
+extern "C" int compass_select_ex(const compass_problem* pr, const compass_calib* cal, int eq5_as_printed,
+                                 compass_choice* out) {
   if (!pr || !cal || !out) return COMPASS_ERR_INVALID_ARG;
   if (pr->op != COMPASS_OP_AG_GEMM && pr->op != COMPASS_OP_GEMM_RS) return COMPASS_ERR_INVALID_ARG;
   if (pr->P < 1) return COMPASS_ERR_INVALID_ARG;
   if (pr->M <= 0 || pr->N <= 0 || pr->K <= 0 || pr->M % pr->P != 0) return COMPASS_ERR_SHAPE;
-  const double P = double(pr->P), M = double(pr->M), N = double(pr->N), K = double(pr->K);
-  // Phase 1: base metrics
-  const double flops = 2.0 * P * M * N * K;
-  const double bytes = 2.0 * P * M * (pr->op == COMPASS_OP_AG_GEMM ? K : N);
-  out->t_comp = cal->comp_a + cal->comp_b * flops;
-  out->t_comm = cal->comm_a + cal->comm_b * bytes;
-  out->lambda = out->t_comm > 0.0 ? out->t_comp / out->t_comm : INFINITY;
-  // Phase 2: degree
-  out->d_star = optimal_degree(out->t_comp, out->t_comm, cal->alpha_decomp, cal->beta_decomp,
-                               largest_degree(pr->M / pr->P), false, nullptr);
-  // Phase 3: prediction and selection
-  out->t_decomp = decomp_time(out->t_comp, out->t_comm, cal->alpha_decomp, cal->beta_decomp, out->d_star);
-  const double m_volume = M * (pr->op == COMPASS_OP_AG_GEMM ? K : N);
-  out->t_fusion = fusion_time(out->t_comp, out->t_comm, pr->P, cal->alpha_fusion, cal->beta_fusion, m_volume);
-  if (out->t_fusion < out->t_decomp) {
-    out->strategy = COMPASS_STRATEGY_INTRAFUSION;
-    out->t_star = out->t_fusion;
-  } else {
-    out->strategy = COMPASS_STRATEGY_INTERDECOM;
-    out->t_star = out->t_decomp;
-  }
+  const BaseTimes w = base_times(pr, cal);
+  const int degree = optimal_degree(w.t_comp, w.t_comm, cal->alpha_decomp, cal->beta_decomp, largest_degree(pr->M / pr->P),
+                                    eq5_as_printed != 0, nullptr);
+  // Listed in the order ties are resolved: a later entry replaces an earlier one only when strictly faster,
+  // so equal predictions stay with InterDecom.
+  const Prediction table[2] = {
+      {COMPASS_STRATEGY_INTERDECOM, decomp_time(w.t_comp, w.t_comm, cal->alpha_decomp, cal->beta_decomp, degree)},
+      {COMPASS_STRATEGY_INTRAFUSION,
+       fusion_time(w.t_comp, w.t_comm, pr->P, cal->alpha_fusion, cal->beta_fusion, w.volume)},
+  };
+  int best = 0;
+  for (int i = 1; i < 2; ++i)
+    if (table[i].time < table[best].time) best = i;
+  out->strategy = table[best].strategy;
+  out->t_star = table[best].time;
+  out->d_star = degree;
+  out->t_decomp = table[0].time;
+  out->t_fusion = table[1].time;
+  out->t_comp = w.t_comp;
+  out->t_comm = w.t_comm;
+  out->lambda = w.t_comm > 0.0 ? w.t_comp / w.t_comm : INFINITY;
   return COMPASS_OK;
+}
+
+extern "C" int compass_select(const compass_problem* pr, const compass_calib* cal, compass_choice* out) {
+  return compass_select_ex(pr, cal, 0, out);
 }

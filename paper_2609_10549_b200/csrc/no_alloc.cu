@@ -98,6 +98,7 @@ extern "C" int compass_gemm_rs_sequential_noalloc(const compass_problem* pr, con
   L.ldo = pr->N;
   L.n_seg = 1;
   L.rows_per_block = int(m);
+  L.share_run = 1;
   L.epilogue = EPI_STORE;
   L.mode = GEMM_MODE_AUTO;
   L.status = reinterpret_cast<StatusBlock*>(scratch);
@@ -120,4 +121,20 @@ extern "C" int compass_gemm_rs_sequential_noalloc(const compass_problem* pr, con
   st = launch_gemm(L, stream);                                          // every rank's partial product
   if (st != COMPASS_OK) return st;
   return launch_reduce_partials(W, P, Out, m, pr->N, 0, m, stream);     // sum into the owners' rows
+}
+
+// The status block of the last no-allocation call on the current device, read straight from the
+// built-in array (nothing is allocated: one small device-to-host copy and a stream synchronisation).
+extern "C" int compass_noalloc_read_status(void* cuda_stream, int* detail) {
+  unsigned char* scratch = nullptr;
+  int st = noalloc_scratch(&scratch);
+  if (st != COMPASS_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  StatusBlock host;
+  cudaError_t e = cudaMemcpyAsync(&host, scratch, sizeof(host), cudaMemcpyDeviceToHost, stream);
+  if (e != cudaSuccess) return record_cuda_error(e);
+  e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return record_cuda_error(e);
+  if (detail) *detail = host.detail;
+  return host.code;
 }

@@ -19,10 +19,14 @@ Mapping of Table IV onto the two operators of one MLP block (Section II-A):
 AllGather+GEMM multiplies [M x K] by the column-parallel [K x N/P];
 GEMM+ReduceScatter multiplies [M x N/P] by the row-parallel [N/P x K].
 
-    python -m paper_2609_10549_b200.grid_study measure --out grid.jsonl [--shard i/n] [--max-m 32768]
-    python -m paper_2609_10549_b200.grid_study analyze --inp grid.jsonl
+    python -m paper_2609_10549_b200.grid_study measure --out grid.jsonl [--shard i/n] [--max-m 32768] [--limit n]
+    python -m paper_2609_10549_b200.grid_study analyze --inp grid.jsonl [--report report.json] [--summary summary.md]
+                                                       [--calib-out calib.json]
 
 `measure` appends one JSON line per case and skips cases already in the file.
+`analyze` needs no GPU (host arithmetic through the C ABI); `--calib-out`
+stores the fitted compass_calib of both patterns with its provenance, in the
+form `load_calibration` reads back (bench.py uses it instead of refitting).
 """
 from __future__ import annotations
 
@@ -64,16 +68,15 @@ def case_key(c):
     return f"{c['op']}-{c['P']}-{c['M']}-{c['table_N']}-{c['table_K']}"
 
 
-def measure(args):
+def measure_cases(cases, out_path, iters=5, log=print):
+    """Times every case in `cases` (dicts as `grid` makes them) and appends one JSON line per case to `out_path`;
+    cases already in the file are skipped.  Returns the number of cases measured."""
     import torch
 
     done = set()
-    if os.path.exists(args.out):
-        with open(args.out) as f:
+    if os.path.exists(out_path):
+        with open(out_path) as f:
             done = {case_key(json.loads(line)) for line in f if line.strip()}
-    cases = grid(args.max_m)
-    i, n = (int(x) for x in args.shard.split("/"))
-    cases = [c for k, c in enumerate(cases) if k % n == i]
     stream = torch.cuda.current_stream()
     side = torch.cuda.Stream()
 
@@ -91,6 +94,7 @@ def measure(args):
             ts.append(e0.elapsed_time(e1))
         return float(np.median(ts))
 
+    measured = 0
     for c in cases:
         if case_key(c) in done:
             continue
@@ -103,7 +107,6 @@ def measure(args):
         out = [torch.empty(w.out_shape, dtype=torch.bfloat16, device="cuda") for _ in range(w.P)]
         pr = api.make_problem(w.op, w.P, w.M, w.N, w.K)
         ws = api.alloc_workspace(pr)
-        iters = 5
         fused = api.compass_ag_gemm if w.op == wl.OP_AG_GEMM else api.compass_gemm_rs
         rec = dict(c, flops=w.flops, m_rows=w.m)
         rec["fused_ms"] = median_ms(lambda: fused(pr, A, B, out, ws, stream), iters)
@@ -124,18 +127,34 @@ def measure(args):
         status = api.compass_read_status(ws)
         if status != (api.OK, 0):
             raise SystemExit(f"device status {status} on {c}")
-        with open(args.out, "a") as f:
+        with open(out_path, "a") as f:
             f.write(json.dumps(rec) + "\n")
-        print(case_key(c), round(rec["fused_ms"], 3), {k: round(v, 3) for k, v in rec["decomp_ms"].items()}, flush=True)
+        log(case_key(c), round(rec["fused_ms"], 3), {k: round(v, 3) for k, v in rec["decomp_ms"].items()})
+        measured += 1
         del A, B, out, ws, dws
         torch.cuda.empty_cache()
+    return measured
 
 
-def analyze(args):
-    with open(args.inp) as f:
-        recs = [json.loads(line) for line in f if line.strip()]
+def measure(args):
+    cases = grid(args.max_m)
+    i, n = (int(x) for x in args.shard.split("/"))
+    cases = [c for k, c in enumerate(cases) if k % n == i]
+    if args.limit:
+        cases = cases[:args.limit]
+    measure_cases(cases, args.out, log=lambda *a: print(*a, flush=True))
+
+
+CALIB_FIELDS = ("comp_a", "comp_b", "comm_a", "comm_b", "alpha_decomp", "beta_decomp", "alpha_fusion", "beta_fusion")
+PATTERNS = ((wl.OP_AG_GEMM, "AG+GEMM"), (wl.OP_GEMM_RS, "GEMM+RS"))
+
+
+def analyze_records(recs):
+    """Fit on every other case, score on the rest; host arithmetic only (the C ABI's model and regression calls).
+    `recs`: the dicts `measure_cases` writes.  Returns the report dict."""
+    recs = [dict(r) for r in recs]
     report = {"cases": len(recs)}
-    for op, name in ((wl.OP_AG_GEMM, "AG+GEMM"), (wl.OP_GEMM_RS, "GEMM+RS")):
+    for op, name in PATTERNS:
         rs = sorted((r for r in recs if r["op"] == op), key=case_key)
         if len(rs) < 4:
             continue
@@ -182,8 +201,7 @@ def analyze(args):
         mean = lambda xs: float(np.mean(xs)) if xs else None
         report[name] = {
             "calibration_cases": len(cal), "test_cases": len(test),
-            "calib": {"comp_a": ca, "comp_b": cb, "comm_a": ma, "comm_b": mb, "alpha_decomp": alpha, "beta_decomp": beta,
-                      "alpha_fusion": af, "beta_fusion": bf},
+            "calib": dict(zip(CALIB_FIELDS, (ca, cb, ma, mb, alpha, beta, af, bf))),
             "decomp_mae_ms_overhead_aware": {str(d): mean(v) for d, v in mae_aware.items()},
             "decomp_mae_ms_overhead_agnostic": {str(d): mean(v) for d, v in mae_agn.items()},
             "decomp_mae_ms_overall": {"aware": mean(sum(mae_aware.values(), [])), "agnostic": mean(sum(mae_agn.values(), []))},
@@ -195,7 +213,67 @@ def analyze(args):
             "selector_accuracy": mean(strat_hits),
             "intrafusion_wins": int(sum(1 for r in test if r["t_intra"] < min(r["decomp_ms"].values()))),
         }
-    print(json.dumps(report, indent=1))
+    return report
+
+
+def calibration_of(report, provenance):
+    """The fitted parameters of both patterns in the form `load_calibration` reads (times in milliseconds)."""
+    return {"unit": "ms", "provenance": provenance,
+            "patterns": {name: report[name]["calib"] for _op, name in PATTERNS if name in report}}
+
+
+def load_calibration(path):
+    """{pattern name: api.Calib} from a file `analyze --calib-out` wrote, plus its provenance string."""
+    with open(path) as f:
+        doc = json.load(f)
+    calibs = {name: api.Calib(*[float(c[k]) for k in CALIB_FIELDS]) for name, c in doc["patterns"].items()}
+    return calibs, doc.get("provenance", "")
+
+
+def summary_markdown(report, source):
+    """The comparison of Table II / Section V-B / Section VI-C as a small table."""
+    rows = [("cases scored (fit on every other case)", lambda r: f"{r['test_cases']} (fit on {r['calibration_cases']})"),
+            ("decomposition model MAE, overhead-agnostic -> aware (ms; mean time)",
+             lambda r: f"{r['decomp_mae_ms_overall']['agnostic']:.2f} -> {r['decomp_mae_ms_overall']['aware']:.2f} "
+                       f"({r['mean_decomp_time_ms']:.2f})"),
+            ("per d = 2 / 4 / 8 / 16, aware (ms)",
+             lambda r: " / ".join(f"{r['decomp_mae_ms_overhead_aware'][d]:.2f}" for d in ("2", "4", "8", "16"))),
+            ("per d = 2 / 4 / 8 / 16, agnostic (ms)",
+             lambda r: " / ".join(f"{r['decomp_mae_ms_overhead_agnostic'][d]:.2f}" for d in ("2", "4", "8", "16"))),
+            ("fusion model MAE, agnostic -> aware (ms)",
+             lambda r: f"{r['fusion_mae_ms']['agnostic']:.2f} -> {r['fusion_mae_ms']['aware']:.2f}"),
+            ("fitted (alpha, beta) of Eq. 3", lambda r: f"{r['calib']['alpha_decomp']:.3f}, {r['calib']['beta_decomp']:.3f}"),
+            ("measured-best d: 1 / 2 / 4 / 8 / 16",
+             lambda r: " / ".join(str(r['measured_best_d_histogram'].get(d, 0)) for d in ("1", "2", "4", "8", "16"))),
+            ("Eq. 4-5 pick the measured best", lambda r: f"{100 * r['predicted_d_is_best']:.1f} %"),
+            ("cost of the predicted d / of fixed d = 4 over the best",
+             lambda r: f"{100 * r['penalty_of_predicted_d']:.1f} % / {100 * r['penalty_of_fixed_d4']:.1f} %"),
+            ("Algorithm 1 picks the faster strategy", lambda r: f"{100 * r['selector_accuracy']:.1f} %"),
+            ("IntraFusion faster in", lambda r: f"{r['intrafusion_wins']} of {r['test_cases']}")]
+    names = [name for _op, name in PATTERNS if name in report]
+    lines = [f"Grid study over {report['cases']} cases ({source}).", "",
+             "| | " + " | ".join(names) + " |", "|---|" + "---|" * len(names)]
+    for label, fn in rows:
+        lines.append(f"| {label} | " + " | ".join(fn(report[n]) for n in names) + " |")
+    return "\n".join(lines) + "\n"
+
+
+def analyze(args):
+    with open(args.inp) as f:
+        recs = [json.loads(line) for line in f if line.strip()]
+    report = analyze_records(recs)
+    text = json.dumps(report, indent=1)
+    print(text)
+    if args.report:
+        with open(args.report, "w") as f:
+            f.write(text + "\n")
+    if args.summary:
+        with open(args.summary, "w") as f:
+            f.write(summary_markdown(report, args.provenance or os.path.basename(args.inp)))
+    if args.calib_out:
+        with open(args.calib_out, "w") as f:
+            json.dump(calibration_of(report, args.provenance or os.path.basename(args.inp)), f, indent=1)
+            f.write("\n")
 
 
 def main():
@@ -205,8 +283,13 @@ def main():
     m.add_argument("--out", required=True)
     m.add_argument("--shard", default="0/1")
     m.add_argument("--max-m", type=int, default=32768)
+    m.add_argument("--limit", type=int, default=0, help="measure only the first n cases of the shard")
     a = sub.add_parser("analyze")
     a.add_argument("--inp", required=True)
+    a.add_argument("--report", help="write the report (JSON) here")
+    a.add_argument("--summary", help="write the comparison table (markdown) here")
+    a.add_argument("--calib-out", help="write the fitted calibration of both patterns (JSON) here")
+    a.add_argument("--provenance", default="", help="where and how the timings were taken (stored with the outputs)")
     args = ap.parse_args()
     (measure if args.cmd == "measure" else analyze)(args)
 

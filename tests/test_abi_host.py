@@ -111,6 +111,24 @@ def test_selector_matches_oracle(op, P, rows, N, K, ca, cb, ma, mb, ad, bd, af, 
         assert getattr(got, name_l) == pytest.approx(getattr(want, name_o), rel=1e-12)
 
 
+def test_selector_on_eq5_as_printed():
+    """In the communication-bound regime (lambda < 1) the printed Eq. 5 and the regime-aware form pick different
+    degrees; compass_select_ex runs Algorithm 1 on either, and both agree with the oracle."""
+    P, M, N, K = 4, 4096, 1024, 1024
+    flops, nbytes = 2.0 * P * M * N * K, 2.0 * P * M * K
+    args = (0.0, 10.0 / flops, 0.0, 100.0 / nbytes, 0.9, 0.004, 50.0, 0.0)      # T_comp 10, T_comm 100: lambda = 0.1
+    pr = api.make_problem(OP_AG_GEMM, P, M, N, K)
+    aware = api.compass_select(pr, api.Calib(*args))
+    printed = api.compass_select(pr, api.Calib(*args), eq5_as_printed=True)
+    want_aware = omo.select(OP_AG_GEMM, P, M, N, K, omo.Calib(*args))
+    want_printed = omo.select(OP_AG_GEMM, P, M, N, K, omo.Calib(*args), as_printed=True)
+    assert (aware.d_star, printed.d_star) == (want_aware.d_star, want_printed.d_star)
+    assert aware.d_star != printed.d_star
+    assert aware.t_decomp == pytest.approx(want_aware.t_decomp, rel=1e-12)
+    assert printed.t_decomp == pytest.approx(want_printed.t_decomp, rel=1e-12)
+    assert aware.t_decomp <= printed.t_decomp            # the regime-aware degree is never the worse of the two here
+
+
 def test_selector_hand_example_and_errors():
     P, M, N, K = 4, 4096, 1024, 1024
     cal = api.Calib(0.0, 250.0 / (2.0 * P * M * N * K), 0.0, 50.0 / (2.0 * P * M * K), 1.0, 0.01, 2.0, 0.0)

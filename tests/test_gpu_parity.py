@@ -4,9 +4,10 @@ on the same seeded inputs.
 Acceptance (every element of every rank's output):
     |gpu - ref| <= 1e-2 * max|ref| + 1e-3         (BF16 output, FP32 accumulate)
 plus RMS error <= 2^-8 of the reference RMS (oracle.compare).  Schedules are
-compared bit-exactly.  Small cases are checked element by element; the
-full-size configurations on a row sample (rows next to every partition and
-tile boundary plus 1 % random rows, full width)."""
+compared bit-exactly.  Every case, the five full-size configurations and all
+their variants (fused, ring read-modify-write, push, InterDecom) included, is
+checked element by element: the FP64 reference of a large configuration is
+computed one rank (or one owner chunk) at a time."""
 import numpy as np
 import pytest
 import torch
@@ -58,6 +59,51 @@ def test_kernel_clock_record_is_plausible():
     assert api.compass_read_status(ws) == (api.OK, 0)
 
 
+def test_tensor_map_cache_serves_repeats_and_misses_on_new_buffers_or_shapes():
+    """The library keeps encoded TMA tensor maps keyed by (pointer, shape, box).  A repeated call on the same
+    buffers must be served from the table; other buffers or another shape must be encoded afresh -- and the
+    results must match the oracle either way (a stale map would read the wrong memory)."""
+    w = small(wl.OP_AG_GEMM, 2, 256, 264, 200, dist=0.1)
+    A_bits, B_bits = wl.make_inputs(w)
+    ref = ops.ag_gemm(A_bits, B_bits)
+    pr = gu.problem_of(w)
+    ws = api.alloc_workspace(pr)
+
+    def run(A, B):
+        outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        api.compass_ag_gemm(pr, A, B, [o.view for o in outs], ws)
+        assert api.compass_read_status(ws) == (api.OK, 0)
+        assert all(o.guards_intact() for o in outs)
+        return [o.bits() for o in outs]
+
+    A, B = gu.device_inputs(A_bits, B_bits)
+    check_all(run(A, B), ref, "first call")
+    h0, m0 = api.tensor_map_cache_stats()
+    check_all(run(A, B), ref, "repeat")
+    h1, m1 = api.tensor_map_cache_stats()
+    assert m1 == m0 and h1 == h0 + 2 * w.P                    # P maps of A and P of B, none encoded again
+    # the same values in other allocations: every map is a new key
+    A2 = [a.clone() for a in A]
+    B2 = [b.clone() for b in B]
+    check_all(run(A2, B2), ref, "new buffers")
+    h2, m2 = api.tensor_map_cache_stats()
+    assert m2 == m1 + 2 * w.P
+    # swapping which rank owns which buffer changes the result; the maps are all known, the answer must follow
+    swapped_ref = ops.ag_gemm(A_bits[::-1], B_bits)
+    check_all(run(A[::-1], B), swapped_ref, "swapped ranks")
+    # another shape on the very same memory: new keys (rows, row length), correct result
+    w2 = small(wl.OP_AG_GEMM, 2, 128, 264, 400, dist=0.1)
+    A_flat = [a.view(-1)[:128 * 400].view(128, 400) for a in A]
+    B_flat = [torch.cat([b.view(-1), b.view(-1)]).view(264, 400) for b in B]
+    bits = lambda ts: [api.to_bits(t.contiguous()) for t in ts]
+    pr2 = gu.problem_of(w2)
+    outs = [gu.Guarded(*w2.out_shape) for _ in range(w2.P)]
+    api.compass_ag_gemm(pr2, A_flat, B_flat, [o.view for o in outs], ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    check_all([o.bits() for o in outs], ops.ag_gemm(bits(A_flat), bits(B_flat)), "same memory, other shape")
+    assert api.tensor_map_cache_stats()[1] > m2
+
+
 def test_config1_ag_gemm_full():
     w = wl.C1_AG
     A, B = wl.make_inputs(w)
@@ -98,6 +144,76 @@ def test_gemm_rs_small_shapes(P, m, N, K, rings):
     outs, status, guards = gu.run_fused(w, A, B, rings=rings)
     assert status == (api.OK, 0) and guards
     check_all(outs, ops.gemm_rs(A, B, rings=rings), w.name)
+
+
+# Partitions below 256 rows: blocks that multiply by the same weight shard are tiled together, a CTA pair taking
+# one 128-row fragment of each of two blocks (the two ring entries of a step; with one ring, consecutive steps of a
+# rank; in InterDecom, consecutive row slices of a rank).  h = 64, 128 and 192 rows, ragged N and K, both launch
+# orders, one and two rings, odd group sizes, all variants; element by element against the oracle.
+SMALL_PARTITION_CASES = [
+    # (P, rows per rank, N, K, rings, order)
+    (4, 256, 520, 200, 2, api.ORDER_RANK_MAJOR), (4, 256, 520, 200, 2, api.ORDER_STEP_MAJOR),
+    (4, 128, 264, 328, 2, api.ORDER_RANK_MAJOR), (8, 384, 776, 72, 2, api.ORDER_STEP_MAJOR),
+    (3, 128, 520, 136, 1, api.ORDER_RANK_MAJOR), (4, 192, 256, 64, 1, api.ORDER_RANK_MAJOR),
+    (5, 100, 264, 200, 1, api.ORDER_STEP_MAJOR), (8, 256, 1032, 456, 2, api.ORDER_RANK_MAJOR),
+    (2, 200, 520, 392, 2, api.ORDER_RANK_MAJOR),
+]
+
+
+@pytest.mark.parametrize("P,m,N,K,rings,order", SMALL_PARTITION_CASES)
+def test_small_partitions_ag_gemm(P, m, N, K, rings, order):
+    w = small(wl.OP_AG_GEMM, P, m, N, K, dist=0.1)
+    A_bits, B_bits = wl.make_inputs(w)
+    pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, rings=rings, order=order)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    ws = api.alloc_workspace(pr)
+    api.compass_ag_gemm(pr, A, B, [o.view for o in outs], ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    assert all(o.guards_intact() for o in outs)
+    check_all([o.bits() for o in outs], ops.ag_gemm(A_bits, B_bits, rings=rings), w.name)
+
+
+@pytest.mark.parametrize("P,m,N,K,rings,order", SMALL_PARTITION_CASES)
+def test_small_partitions_ring_rmw_and_segmented(P, m, N, K, rings, order):
+    w = small(wl.OP_GEMM_RS, P, m, N, K, dist=0.05)
+    A, B = wl.make_inputs(w)
+    ref = ops.gemm_rs(A, B, rings=rings)
+    outs, status, guards = gu.run_fused(w, A, B, rings=rings, rs_variant=api.RS_RING_RMW)
+    assert status == (api.OK, 0) and guards
+    check_ring(outs, ref, w.name, P)
+    outs, status, guards = gu.run_fused(w, A, B, rings=rings)
+    assert status == (api.OK, 0) and guards
+    check_all(outs, ref, w.name)
+
+
+def test_small_partitions_ring_rmw_integers_exact_and_counters_return_to_zero():
+    w = wl.Workload("ints-ring-small", wl.OP_GEMM_RS, P=4, M=4 * 256, N=520, K=64)      # h = 128: one fragment per partition
+    A_bits, B_bits = wl.make_structured_inputs(w, "index")
+    pr = gu.problem_of(w, rs_variant=api.RS_RING_RMW)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    ws = api.alloc_workspace(pr)
+    ref = ops.gemm_rs(A_bits, B_bits)
+    for _ in range(2):
+        outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        api.compass_gemm_rs(pr, A, B, [o.view for o in outs], ws)
+        assert api.compass_read_status(ws) == (api.OK, 0)
+        for o, r in zip(outs, ref):
+            assert np.array_equal(ops.bf16_bits_to_f64(o.bits()), r)
+        assert int(ws[api.STATUS_BYTES:].view(torch.int32).abs().sum().item()) == 0
+
+
+@pytest.mark.parametrize("op,P,m,N,K,d", [
+    (wl.OP_AG_GEMM, 4, 1024, 520, 200, 8), (wl.OP_AG_GEMM, 4, 1024, 520, 200, 16), (wl.OP_AG_GEMM, 3, 384, 264, 72, 2),
+    (wl.OP_GEMM_RS, 4, 1024, 520, 200, 8), (wl.OP_GEMM_RS, 4, 1024, 520, 200, 16), (wl.OP_GEMM_RS, 5, 512, 264, 72, 4),
+])
+def test_small_slices_interdecom(op, P, m, N, K, d):
+    w = small(op, P, m, N, K, dist=0.1)
+    A, B = wl.make_inputs(w)
+    refs = ops.decomp_ag_gemm(A, B, d) if op == wl.OP_AG_GEMM else ops.decomp_gemm_rs(A, B, d)
+    outs, status, guards = gu.run_decomp(w, A, B, d)
+    assert status == (api.OK, 0) and guards
+    check_all(outs, refs, f"{w.name} d={d}")
 
 
 # Enough 512-row partitions to fill whole waves of CTA pairs with 512x256 tiles and leave a
@@ -144,72 +260,81 @@ def test_integer_inputs_are_reproduced_exactly(op):
         assert np.array_equal(ops.bf16_bits_to_f64(got), ops.f64_to_bf16_f64(ref))
 
 
-def _sampled_ag(w, rings=2):
-    A, B = wl.make_inputs(w)
-    outs, status, guards = gu.run_fused(w, A, B, rings=rings)
-    assert status == (api.OK, 0) and guards
-    rows = gu.sample_rows(w.M, w.P, rings)
-    refs = ops.ag_gemm(A, B, rings=rings, rows=rows)
+# ---- the five configurations at full size, every element of every rank ---------------------------------
+
+_REF_CACHE = {}
+
+
+def _inputs(w):
+    key = ("in", w.op, w.P, w.M, w.N, w.K, w.a_dist, w.b_dist, w.seed)
+    if key not in _REF_CACHE:
+        _REF_CACHE[key] = wl.make_inputs(w)
+    return _REF_CACHE[key]
+
+
+def _reference(w, idx, cache):
+    """FP64 reference of rank `idx` (AllGather+GEMM) or owner chunk `idx` (GEMM+ReduceScatter) of workload w.
+    Configurations 2 and 4 share their AllGather+GEMM inputs, and several variants are checked against the
+    same reference, so the smaller ones are kept."""
+    key = ("ref", w.op, w.P, w.M, w.N, w.K, w.a_dist, w.b_dist, w.seed, idx)
+    if key in _REF_CACHE:
+        return _REF_CACHE[key]
+    A, B = _inputs(w)
+    (ref,) = ops.ag_gemm(A, B, ranks=[idx]) if w.op == wl.OP_AG_GEMM else ops.gemm_rs(A, B, chunks=[idx])
+    if cache:
+        _REF_CACHE[key] = ref
+    return ref
+
+
+def check_every_element(w, outs, what, ring_rmw=False, one_rounding=True, cache=True, block_rows=2048):
+    """All elements of all P outputs against the oracle.  The comparison runs over row blocks (its FP64
+    temporaries stay small) with max|ref| taken over the rank's whole tensor, as the acceptance rule says."""
+    rms_limit = 2.0 ** -9 * max(1.0, w.P ** 0.5) if ring_rmw else compare.RMS_REL_LIMIT
     for r in range(w.P):
-        assert not np.any((outs[r] & 0x7F80) == 0x7F80), "NaN/Inf or unwritten output"
-        rep = compare.check(outs[r][rows], refs[r])
-        assert rep.ok, f"{w.name} rank {r}: {rep}"
+        ref = _reference(w, r, cache)
+        assert outs[r].shape == ref.shape
+        max_ref = float(np.max(np.abs(ref)))
+        within, n = 0.0, 0
+        for lo in range(0, ref.shape[0], block_rows):
+            rep = compare.check(outs[r][lo:lo + block_rows], ref[lo:lo + block_rows], max_ref=max_ref)
+            assert rep.violations == 0 and rep.rms_rel <= rms_limit, f"{what} rank/chunk {r} rows {lo}+: {rep}"
+            rows = ref[lo:lo + block_rows].shape[0]
+            within += rep.frac_within_1ulp * rows
+            n += rows
+        # FP32 accumulation and one rounding: almost every element is the correctly rounded BF16 or its neighbour.
+        # The exceptions are results that nearly cancel: the FP32 sum of K terms carries an absolute error of about
+        # sqrt(K) * 2^-24 of the typical magnitude, which exceeds a BF16 step only for elements below ~2^-9 of it
+        # (a fraction of about 0.1 % at K = 28672, the longest contraction here).
+        if one_rounding and not ring_rmw:
+            assert within / n > 0.997, f"{what} rank/chunk {r}: only {within / n:.5f} of the elements within one BF16 step"
+        del ref
 
 
-def _sampled_rs(w, rings=2, rs_variant=api.RS_SEGMENTED_K):
-    A, B = wl.make_inputs(w)
-    outs, status, guards = gu.run_fused(w, A, B, rings=rings, rs_variant=rs_variant)
-    assert status == (api.OK, 0) and guards
-    rows = gu.sample_rows(w.M, w.P, rings)
-    found = ops.gemm_rs_rows(A, B, rows, rings=rings)
-    assert sorted(found) == list(range(w.P))
-    for c, (local, ref) in found.items():
-        assert not np.any((outs[c] & 0x7F80) == 0x7F80), "NaN/Inf or unwritten output"
-        rep = compare.check(outs[c][local], ref)
-        assert rep.ok, f"{w.name} chunk {c}: {rep}"
+def _drop_cached(w):
+    for key in [k for k in _REF_CACHE if k[1:9] == (w.op, w.P, w.M, w.N, w.K, w.a_dist, w.b_dist, w.seed)]:
+        del _REF_CACHE[key]
 
 
-def test_config2_ag_gemm_full_size_sampled():
-    _sampled_ag(wl.C2_AG)
-
-
-def test_config3_gemm_rs_full_size_sampled():
-    _sampled_rs(wl.C3_RS)
-
-
-def test_config4_gemm_rs_full_size_sampled():
-    _sampled_rs(wl.C4_RS)
-
-
-# The two operators of the benchmark step, in the configuration bench.py times, every element of every rank.
-def test_config2_ag_gemm_every_element():
-    w = wl.C2_AG
-    A, B = wl.make_inputs(w)
+@pytest.mark.parametrize("w", [wl.C2_AG, wl.C3_RS, wl.C4_RS], ids=lambda w: w.name)
+def test_fused_every_element(w):
+    """Configurations 2, 3 (the operators bench.py times, in the configuration it times) and the
+    GEMM+ReduceScatter of configuration 4."""
+    A, B = _inputs(w)
     outs, status, guards = gu.run_fused(w, A, B)
     assert status == (api.OK, 0) and guards
-    for r in range(w.P):                                   # one rank at a time keeps the FP64 reference at 100 MB
-        (ref,) = ops.ag_gemm(A, B, ranks=[r])
-        rep = compare.check(outs[r], ref)
-        assert rep.ok and rep.frac_within_1ulp > 0.999, f"{w.name} rank {r}: {rep}"
+    check_every_element(w, outs, w.name)
 
 
-def test_config3_gemm_rs_every_element():
-    w = wl.C3_RS
-    A, B = wl.make_inputs(w)
+@pytest.mark.parametrize("w", [wl.C5_AG, wl.C5_RS], ids=lambda w: w.name)
+def test_config5_fused_every_element(w):
+    """The 70B-class pair: 1.5e13 and 7.7e12 FLOP of FP64 reference, one rank / owner chunk at a time."""
+    A, B = _inputs(w)
     outs, status, guards = gu.run_fused(w, A, B)
     assert status == (api.OK, 0) and guards
-    for c in range(w.P):
-        (ref,) = ops.gemm_rs(A, B, chunks=[c])
-        rep = compare.check(outs[c], ref)
-        assert rep.ok and rep.frac_within_1ulp > 0.999, f"{w.name} chunk {c}: {rep}"
-
-
-def test_config5_ag_gemm_full_size_sampled():
-    _sampled_ag(wl.C5_AG)
-
-
-def test_config5_gemm_rs_full_size_sampled():
-    _sampled_rs(wl.C5_RS)
+    try:
+        check_every_element(w, outs, w.name, cache=False)
+    finally:
+        _drop_cached(w)
 
 
 @pytest.mark.parametrize("op,P,m,N,K,d", [
@@ -229,21 +354,13 @@ def test_interdecom_small_shapes(op, P, m, N, K, d):
 
 
 @pytest.mark.parametrize("d", [1, 4, 16])
-def test_config4_interdecom_full_size_sampled(d):
-    for w in (wl.C4_AG, wl.C4_RS):
-        A, B = wl.make_inputs(w)
-        outs, status, guards = gu.run_decomp(w, A, B, d)
-        assert status == (api.OK, 0) and guards
-        rows = gu.sample_rows(w.M, w.P, 2, tile=max(1, w.m // d))
-        if w.op == wl.OP_AG_GEMM:
-            refs = ops.ag_gemm(A, B, rows=rows)
-            for r in range(w.P):
-                rep = compare.check(outs[r][rows], refs[r])
-                assert rep.ok, f"{w.name} d={d} rank {r}: {rep}"
-        else:
-            for c, (local, ref) in ops.gemm_rs_rows(A, B, rows).items():
-                rep = compare.check(outs[c][local], ref)
-                assert rep.ok, f"{w.name} d={d} chunk {c}: {rep}"
+@pytest.mark.parametrize("w", [wl.C4_AG, wl.C4_RS], ids=lambda w: w.name)
+def test_config4_interdecom_every_element(w, d):
+    A, B = _inputs(w)
+    outs, status, guards = gu.run_decomp(w, A, B, d)
+    assert status == (api.OK, 0) and guards
+    # the decomposed GEMM+ReduceScatter rounds every rank's partial to BF16 before the reduce kernel adds them
+    check_every_element(w, outs, f"{w.name} d={d}", one_rounding=w.op == wl.OP_AG_GEMM)
 
 
 @pytest.mark.parametrize("op", [wl.OP_AG_GEMM, wl.OP_GEMM_RS])
@@ -308,15 +425,12 @@ def test_ring_rmw_integers_exact_and_counters_return_to_zero():
         assert int(ws[api.STATUS_BYTES:].view(torch.int32).abs().sum().item()) == 0
 
 
-def test_config3_ring_rmw_full_size_sampled():
+def test_config3_ring_rmw_every_element():
     w = wl.C3_RS
-    A, B = wl.make_inputs(w)
+    A, B = _inputs(w)
     outs, status, guards = gu.run_fused(w, A, B, rs_variant=api.RS_RING_RMW)
     assert status == (api.OK, 0) and guards
-    rows = gu.sample_rows(w.M, w.P, 2)
-    for c, (local, ref) in ops.gemm_rs_rows(A, B, rows).items():
-        rep = compare.check(outs[c][local], ref)
-        assert rep.violations == 0 and rep.rms_rel <= 2.0 ** -9 * w.P ** 0.5, f"{w.name} chunk {c}: {rep}"
+    check_every_element(w, outs, f"{w.name} ring-RMW", ring_rmw=True)
 
 
 def test_bounded_wait_reports_timeout_and_the_context_survives():
@@ -370,7 +484,8 @@ def run_push(w, A_bits, B_bits, rings=2, calls=1):
 
 @pytest.mark.parametrize("P,m,N,K,rings", [
     (1, 256, 256, 64, 2), (2, 256, 256, 256, 2), (2, 144, 264, 72, 2), (3, 272, 520, 344, 2), (4, 512, 768, 512, 2),
-    (4, 384, 1024, 320, 1), (8, 256, 512, 192, 2), (4, 1024, 2568, 200, 2),
+    (4, 384, 1024, 320, 1), (8, 256, 512, 192, 2), (4, 1024, 2568, 200, 2), (4, 256, 520, 200, 2), (4, 128, 264, 72, 2),
+    (3, 384, 264, 136, 2),
 ])
 def test_ag_gemm_push_small_shapes(P, m, N, K, rings):
     w = small(wl.OP_AG_GEMM, P, m, N, K, dist=0.1)
@@ -388,16 +503,43 @@ def test_ag_gemm_push_repeated_calls_share_a_workspace():
         check_all(outs, ref, w.name)
 
 
-def test_config2_ag_gemm_push_full_size_sampled():
+def test_push_flag_wait_reports_timeout_and_the_context_survives():
+    """A readiness flag that is never raised (the host leaves out one flag write: a lost message) makes the
+    tile that needs the partition give up after the wait limit: the status must read COMPASS_ERR_TIMEOUT at
+    the readiness-flag wait, the kernel must return, and the next call on the same workspace must be correct."""
+    w = small(wl.OP_AG_GEMM, 4, 512, 520, 200, dist=0.1)
+    A_bits, B_bits = wl.make_inputs(w)
+    pr = gu.problem_of(w)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    ws = torch.empty(api.compass_workspace_bytes(pr, api.WS_PUSH), dtype=torch.uint8, device="cuda")
+    api.compass_workspace_init(ws)
+    side = torch.cuda.Stream()
+    outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    torch.cuda.synchronize()
+    api.compass_set_wait_limit_us(20000)
+    api.compass_test_drop_flag_writes(1)
+    try:
+        api.compass_ag_gemm_push(pr, A, B, [o.view for o in outs], ws, torch.cuda.current_stream(), side)
+        status, detail = api.compass_read_status(ws)
+    finally:
+        api.compass_test_drop_flag_writes(0)
+        api.compass_set_wait_limit_us(0)
+    torch.cuda.synchronize()
+    assert status == api.ERR_TIMEOUT and detail == 7          # the readiness-flag wait
+    assert all(o.guards_intact() for o in outs)
+    api.compass_workspace_init(ws)
+    outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    api.compass_ag_gemm_push(pr, A, B, [o.view for o in outs], ws, torch.cuda.current_stream(), side)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    torch.cuda.synchronize()
+    check_all([o.bits() for o in outs], ops.ag_gemm(A_bits, B_bits), w.name)
+
+
+def test_config2_ag_gemm_push_every_element():
     w = wl.C2_AG
-    A, B = wl.make_inputs(w)
+    A, B = _inputs(w)
     (outs,) = run_push(w, A, B)
-    rows = gu.sample_rows(w.M, w.P, 2)
-    refs = ops.ag_gemm(A, B, rows=rows)
-    for r in range(w.P):
-        assert not np.any((outs[r] & 0x7F80) == 0x7F80), "NaN/Inf or unwritten output"
-        rep = compare.check(outs[r][rows], refs[r])
-        assert rep.ok, f"{w.name} rank {r}: {rep}"
+    check_every_element(w, outs, f"{w.name} push")
 
 
 # ---- invariances: the same arithmetic in the same k order must give the same bits ------------------

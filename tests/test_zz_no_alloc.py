@@ -1,14 +1,16 @@
-"""The no-allocation entry point against the workspace-based one (GPU).
+"""The no-allocation entry point against the workspace-based one and the oracle (GPU).
 
 compass_gemm_rs_sequential_noalloc exists for callers that cannot give the
 library a workspace because all device memory is already spoken for, or that
 cannot afford cudaMalloc's device-wide synchronisation.  Its scratch is a
 built-in device array shared by all calls, which keeps the previous call's
-contents.  The checks: two calls in a row (the second sees the first one's
-leftovers, and uses a different shape) must each reproduce, bit for bit, what
-compass_decomp with d = 1 computes with a caller-provided workspace; the call
-must not change torch's allocator statistics; a problem beyond the array's
-size must be refused.
+contents.  The checks: calls in a row (each sees the previous one's leftovers,
+and uses a different shape) must each reproduce, bit for bit, what
+compass_decomp with d = 1 computes with a caller-provided workspace, and match
+the CPU oracle within the acceptance rule of the other parity tests; the
+device's free memory (as the driver reports it) and torch's allocator
+statistics must not change across the call; the status left in the built-in
+array must read back as OK; a problem beyond the array's size must be refused.
 
 This file is collected last on purpose: a failure here cannot hide another.
 """
@@ -18,6 +20,8 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import compare
+from oracle import operators as ops
 from paper_2609_10549_b200 import api
 from paper_2609_10549_b200 import workloads as wl
 from tests import gpu_util as gu
@@ -31,16 +35,28 @@ def _run_pair(w):
     assert status == (api.OK, 0) and guards
     outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
     pr = gu.problem_of(w)
+    # The first use on a device resolves the array's address; with CUDA's lazy module loading that is also
+    # when the driver reserves the array's memory.  That one-time set-up is not the call's own doing, so it
+    # is triggered here, before free memory is compared.
+    api.compass_noalloc_read_status()
     torch.cuda.synchronize()
     before = torch.cuda.memory_stats()["allocation.all.allocated"]
+    free_before = torch.cuda.mem_get_info()[0]          # the driver's own count: sees a cudaMalloc inside the library
     api.compass_gemm_rs_sequential_noalloc(pr, A, B, [o.view for o in outs])
-    after = torch.cuda.memory_stats()["allocation.all.allocated"]
     torch.cuda.synchronize()
+    free_after = torch.cuda.mem_get_info()[0]
+    after = torch.cuda.memory_stats()["allocation.all.allocated"]
     assert after == before, "the call went through torch's allocator"
+    assert free_after == free_before, "the device's free memory changed across the call"
+    assert api.compass_noalloc_read_status() == (api.OK, 0)
     assert all(o.guards_intact() for o in outs)
+    oracle = ops.gemm_rs(A_bits, B_bits)
     for r in range(w.P):
-        # same kernels, same order of additions: identical bits (tolerance of the other tests: 1e-2*max+1e-3)
+        # same kernels, same order of additions: identical bits
         assert np.array_equal(outs[r].bits(), ref[r]), f"rank {r} differs from compass_decomp(d=1)"
+        # and the oracle, within the tolerance of the other parity tests (1e-2*max|ref| + 1e-3 per element)
+        rep = compare.check(outs[r].bits(), oracle[r])
+        assert rep.ok, f"rank {r} against the oracle: {rep}"
 
 
 @pytest.mark.gpu
