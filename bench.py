@@ -36,9 +36,12 @@ UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes (read + written) per launch of the GEMM kernel, from an ncu capture of
-# `bench.py --steps 1 --warmup 3 --no-cpu-baseline --no-sweep` (dram__bytes_read.sum + dram__bytes_write.sum).
-NCU_TRAFFIC_BYTES = {"C2": 362.6e6, "C3": 799.0e6}
+# DRAM bytes (read + written) per launch of the GEMM kernel: dram__bytes_read.sum + dram__bytes_write.sum of one
+# ncu capture of `bench.py --steps 1 --warmup 3 --no-cpu-baseline --no-sweep`; the summary that holds the figures is
+# named beside them.  They are constants of that capture, not something this run measures.
+NCU_TRAFFIC = {"C2": {"bytes": 362.6e6, "source": "profiles/gemm_mixed_kernel_C2_C3.md"},
+               "C3": {"bytes": 799.0e6, "source": "profiles/gemm_mixed_kernel_C2_C3.md"}}
+CALIBRATION_FILE = os.path.join(ROOT, "paper_2609_10549_b200", "calibration", "calib_b200.json")
 
 
 def env_int(name, default):
@@ -306,7 +309,18 @@ def mlp_report(torch, api):
             "kernels_per_call": 2, "intermediate_bytes": 2 * w.P * w.M * w.hc}
 
 
-def interdecom_report(torch, api, hbm_gbs):
+def stored_calibration(api):
+    """The calibration the grid study wrote (one-time offline regression, Section IV-C), or None."""
+    if not os.path.exists(CALIBRATION_FILE):
+        return None
+    from paper_2609_10549_b200 import grid_study
+    calibs, provenance = grid_study.load_calibration(CALIBRATION_FILE)
+    if "AG+GEMM" not in calibs or "GEMM+RS" not in calibs:
+        return None
+    return calibs["AG+GEMM"], calibs["GEMM+RS"], provenance
+
+
+def interdecom_report(torch, api, hbm_gbs, recalibrate=False):
     """Times compass_decomp for d in {1,2,4,8,16} on the config-4 shapes, fits
     the models' parameters on other shapes (Section IV-C: one-time offline
     regression), and sets the measured-best degree and strategy beside the
@@ -329,6 +343,25 @@ def interdecom_report(torch, api, hbm_gbs):
             ts.append(e0.elapsed_time(e1))
         return float(np.median(ts))
 
+    def interleaved_ms(fns, iters=8, warm=2):
+        """Median time of every callable in `fns`, the variants timed in turn inside one loop: the board's
+        power state (which sets the clock of these tensor-bound kernels) drifts over hundreds of milliseconds, so
+        variants timed one after the other would not be compared at the same clock."""
+        for _ in range(warm):
+            for fn in fns.values():
+                fn()
+        torch.cuda.synchronize()
+        ts = {k: [] for k in fns}
+        for _ in range(iters):
+            for k, fn in fns.items():
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                fn()
+                e1.record(stream)
+                torch.cuda.synchronize()
+                ts[k].append(e0.elapsed_time(e1))
+        return {k: float(np.median(v)) for k, v in ts.items()}
+
     class Case:
         def __init__(self, w):
             self.w = w
@@ -344,21 +377,30 @@ def interdecom_report(torch, api, hbm_gbs):
             self.dws = None
             self.pws = None
 
-        def t_fused(self):
-            return median_ms(lambda: self.fused(self.pr, self.A, self.B, self.out, self.ws, stream))
+        def fn_fused(self):
+            return lambda: self.fused(self.pr, self.A, self.B, self.out, self.ws, stream)
 
-        def t_push(self):
+        def fn_push(self):
             """AllGather+GEMM with pushed partitions and readiness flags (the paper's mechanism)."""
             if self.pws is None:
                 self.pws = torch.empty(api.compass_workspace_bytes(self.pr, api.WS_PUSH), dtype=torch.uint8, device="cuda")
                 api.compass_workspace_init(self.pws)
-            return median_ms(lambda: api.compass_ag_gemm_push(self.pr, self.A, self.B, self.out, self.pws, stream, side))
+            return lambda: api.compass_ag_gemm_push(self.pr, self.A, self.B, self.out, self.pws, stream, side)
 
-        def t_decomp(self, d):
+        def fn_decomp(self, d):
             pr = api.make_problem(self.w.op, self.w.P, self.w.M, self.w.N, self.w.K, d=d)
             if self.dws is None:
                 self.dws = api.alloc_workspace(pr, api.WS_DECOMP)
-            return median_ms(lambda: api.compass_decomp(pr, self.A, self.B, self.out, self.dws, stream, side))
+            return lambda: api.compass_decomp(pr, self.A, self.B, self.out, self.dws, stream, side)
+
+        def t_fused(self):
+            return median_ms(self.fn_fused())
+
+        def t_push(self):
+            return median_ms(self.fn_push())
+
+        def t_decomp(self, d):
+            return median_ms(self.fn_decomp(d))
 
         def volume(self):
             return float(self.w.M) * (self.w.K if self.w.op == wl.OP_AG_GEMM else self.w.N)
@@ -397,10 +439,15 @@ def interdecom_report(torch, api, hbm_gbs):
     def predict_and_measure(w, calib, measure_all):
         c = Case(w)
         choice = api.compass_select(c.pr, calib)
-        t_fused = c.t_fused()
-        t_push = c.t_push() if w.op == wl.OP_AG_GEMM else None
         ds = [d for d in degrees if w.m % d == 0] if measure_all else sorted({1, choice.d_star})
-        times = {d: c.t_decomp(d) for d in ds}
+        fns = {"fused": c.fn_fused()}
+        if w.op == wl.OP_AG_GEMM:
+            fns["push"] = c.fn_push()
+        for d in ds:
+            fns[d] = c.fn_decomp(d)
+        ms = interleaved_ms(fns)            # all variants in turn inside one loop: compared at the same board state
+        t_fused, t_push = ms["fused"], ms.get("push")
+        times = {d: ms[d] for d in ds}
         best_d = min(times, key=times.get)
         # IntraFusion as the paper builds it moves the partitions while it computes: compare that variant with
         # InterDecom where it exists; the gather-by-address kernel (no transfers at all) is reported beside it.
@@ -418,6 +465,7 @@ def interdecom_report(torch, api, hbm_gbs):
                              "gbs": phase_bytes / (phase_ms * 1e-3) / 1e9,
                              "frac_of_measured_hbm": phase_bytes / (phase_ms * 1e-3) / 1e9 / hbm_gbs,
                              "how": "T_decomp(d=1) - T_fused: the phase runs strictly before (gather) or after (reduce) the GEMM"},
+               "timing": "median of 8 rounds; every round times each variant once, in turn",
                "decomp_ms": {str(d): t for d, t in times.items()},
                "measured_best_d": best_d, "predicted_d": choice.d_star,
                "predicted_strategy": "IntraFusion" if choice.strategy == api.STRATEGY_INTRAFUSION else "InterDecom",
@@ -428,17 +476,23 @@ def interdecom_report(torch, api, hbm_gbs):
         torch.cuda.empty_cache()
         return out
 
-    cal_ag = calibrate([wl.Workload("cal-AG-a", wl.OP_AG_GEMM, P=4, M=2048, N=3072, K=4096),
-                        wl.Workload("cal-AG-b", wl.OP_AG_GEMM, P=4, M=8192, N=2048, K=4096),
-                        wl.Workload("cal-AG-c", wl.OP_AG_GEMM, P=8, M=8192, N=2048, K=8192)])
-    cal_rs = calibrate([wl.Workload("cal-RS-a", wl.OP_GEMM_RS, P=4, M=2048, N=4096, K=1024),
-                        wl.Workload("cal-RS-b", wl.OP_GEMM_RS, P=4, M=8192, N=2048, K=1024),
-                        wl.Workload("cal-RS-c", wl.OP_GEMM_RS, P=8, M=8192, N=4096, K=1024)])
+    stored = None if recalibrate else stored_calibration(api)
+    if stored is not None:
+        cal_ag, cal_rs, provenance = stored
+        source = f"loaded from {os.path.relpath(CALIBRATION_FILE, ROOT)}: {provenance}"
+    else:
+        cal_ag = calibrate([wl.Workload("cal-AG-a", wl.OP_AG_GEMM, P=4, M=2048, N=3072, K=4096),
+                            wl.Workload("cal-AG-b", wl.OP_AG_GEMM, P=4, M=8192, N=2048, K=4096),
+                            wl.Workload("cal-AG-c", wl.OP_AG_GEMM, P=8, M=8192, N=2048, K=8192)])
+        cal_rs = calibrate([wl.Workload("cal-RS-a", wl.OP_GEMM_RS, P=4, M=2048, N=4096, K=1024),
+                            wl.Workload("cal-RS-b", wl.OP_GEMM_RS, P=4, M=8192, N=2048, K=1024),
+                            wl.Workload("cal-RS-c", wl.OP_GEMM_RS, P=8, M=8192, N=4096, K=1024)])
+        source = "fitted in this run on three shapes per pattern, none of them predicted below"
     fields = ("comp_a", "comp_b", "comm_a", "comm_b", "alpha_decomp", "beta_decomp", "alpha_fusion", "beta_fusion")
     return {
         "calibration": {"unit": "ms", "AG": {f: getattr(cal_ag, f) for f in fields},
                         "RS": {f: getattr(cal_rs, f) for f in fields},
-                        "shapes": "three shapes per pattern, none of them predicted below"},
+                        "source": source},
         "config4": [predict_and_measure(wl.C4_AG, cal_ag, True), predict_and_measure(wl.C4_RS, cal_rs, True)],
         "config5": [predict_and_measure(wl.C5_AG, cal_ag, True), predict_and_measure(wl.C5_RS, cal_rs, True)],
         "paper_context": "paper (8x RTX A6000, hybrid NVLink-PCIe): IntraFusion 1.5-2.5x over sequential, InterDecom up to "
@@ -507,13 +561,17 @@ def run_ours(args, w_ag, w_rs):
             self.call(self.pr, self.A, self.B, self.out, self.ws, stream)
 
     ag, rs = Op(w_ag), Op(w_rs)
-    calib = api.Calib(0.0, 1.0 / 1.2e15, 0.0, 1.0 / 3.0e12, 1.0, 0.02, 2e-6, 0.0)   # replaced by the sweep's fit below
+    stored = stored_calibration(api)
+    if stored is not None:
+        calib_ag, calib_rs = stored[0], stored[1]
+    else:       # no stored calibration: nominal rates (times in ms), enough for the selector call of the step
+        calib_ag = calib_rs = api.Calib(0.0, 1.0 / 1.2e12, 0.0, 1.0 / 3.0e9, 1.0, 0.02, 2e-3, 0.0)
 
     def step(ev=None):
         api.compass_schedule(w_ag.op, w_ag.P, 2, w_ag.M)
         api.compass_schedule(w_rs.op, w_rs.P, 2, w_rs.M)
-        api.compass_select(ag.pr, calib)
-        api.compass_select(rs.pr, calib)
+        api.compass_select(ag.pr, calib_ag)
+        api.compass_select(rs.pr, calib_rs)
         if ev is not None:
             ev[0].record(stream)
         ag.run()
@@ -577,8 +635,8 @@ def run_ours(args, w_ag, w_rs):
     def e2e_step():
         api.compass_schedule(w_ag.op, w_ag.P, 2, w_ag.M)
         api.compass_schedule(w_rs.op, w_rs.P, 2, w_rs.M)
-        api.compass_select(ag.pr, calib)
-        api.compass_select(rs.pr, calib)
+        api.compass_select(ag.pr, calib_ag)
+        api.compass_select(rs.pr, calib_rs)
         hag.run(s_ag)
         hrs.run(s_rs)
 
@@ -613,19 +671,53 @@ def run_ours(args, w_ag, w_rs):
         achieved = (flops_step / 2.0) / kernel_s / 1e12
         sustained = total_ms >= 1000.0
         peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
-        traffic = None
-        if NCU_TRAFFIC_BYTES:
-            traffic = (NCU_TRAFFIC_BYTES["C2"] + NCU_TRAFFIC_BYTES["C3"]) / 2.0
+        traffic = (NCU_TRAFFIC["C2"]["bytes"] + NCU_TRAFFIC["C3"]["bytes"]) / 2.0     # per launch, like `achieved`
+        protocol = None
+        h2d_bytes, d2h_bytes = hag.h2d + hrs.h2d, hag.d2h + hrs.d2h
+        if world == 1 and not args.no_sweep:
+            del hag, hrs
+            torch.cuda.empty_cache()
+            protocol = timing_protocol_report(torch, api, {"ag_gemm": ag, "gemm_rs": rs})
+
+        def operator_roofline(key, w, t_ms, traffic_key):
+            """One fused operator against both measured peaks: its mean launch inside the timed region (a burst
+            when the region is short) over the burst cuBLAS peak, and its 2 s back-to-back loop over the
+            sustained cuBLAS peak."""
+            tf = w.flops / (t_ms * 1e-3) / 1e12
+            tr = NCU_TRAFFIC[traffic_key]
+            out = {"kernel": "gemm_mixed_kernel", "flops_per_launch": w.flops, "algorithmic_bytes": w.algorithmic_bytes,
+                   "ms": t_ms, "achieved": tf, "unit": UNIT,
+                   "burst": {"tflops": tf, "peak": peaks["bf16_tflops"], "frac": tf / peaks["bf16_tflops"],
+                             "timed": f"mean of {args.steps} launches inside the timed region"},
+                   "sustained": None,
+                   "frac_of_nominal_2250": tf / NOMINAL_BF16_TFLOPS,
+                   "hbm_time_bound_ms": w.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3,
+                   "traffic": tr["bytes"], "traffic_source": tr["source"],
+                   "traffic_over_algorithmic": tr["bytes"] / w.algorithmic_bytes}
+            if protocol is not None:
+                sus = protocol[key]["sustained"]
+                out["sustained"] = {"tflops": sus["tflops"], "peak": peaks["bf16_tflops_sustained"],
+                                    "frac": sus["tflops"] / peaks["bf16_tflops_sustained"],
+                                    "timed": f"{sus['launches']} launches back to back, {sus['seconds']:.1f} s",
+                                    "kernel_sm_mhz": sus["kernel_sm_mhz"]}
+                alone = protocol[key]["alone"]
+                out["alone"] = {"tflops": alone["tflops_median"], "frac_of_burst_peak": alone["tflops_median"] / peaks["bf16_tflops"],
+                                "timed": "median of 100 launches, a synchronisation after each"}
+            return out
+
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(w_ag, w_rs),
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                          "frac": achieved / peak, "traffic": traffic,
-                         "peak_source": f"{'sustained' if sustained else 'burst'} cuBLAS bf16, of {peak_src}",
+                         "peak_source": f"{'sustained' if sustained else 'burst'} cuBLAS bf16, of {peak_src} "
+                                        f"(the timed region lasts {total_ms:.0f} ms)",
                          "kernel": "gemm_mixed_kernel (two launches per step: AG-GEMM and GEMM-RS)",
-                         "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
-                         "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS},
+                         "traffic_source": "mean of the two operators' launches, " + NCU_TRAFFIC["C2"]["source"],
+                         "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
+                         "per_operator": {"C2_ag_gemm": operator_roofline("ag_gemm", w_ag, t_ag, "C2"),
+                                          "C3_gemm_rs": operator_roofline("gemm_rs", w_rs, t_rs, "C3")}},
             "ag_gemm": {"ms": t_ag, "ms_median": float(np.median(ag_ms)), "ms_best": float(np.min(ag_ms)),
                         "tflops": w_ag.flops / (t_ag * 1e-3) / 1e12,
                         "frac_of_nominal_2250": w_ag.flops / (t_ag * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS},
@@ -633,19 +725,17 @@ def run_ours(args, w_ag, w_rs):
                         "tflops": w_rs.flops / (t_rs * 1e-3) / 1e12,
                         "frac_of_nominal_2250": w_rs.flops / (t_rs * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS},
             "e2e": {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
-                    "h2d_bytes_per_step": hag.h2d + hrs.h2d, "d2h_bytes_per_step": hag.d2h + hrs.d2h,
+                    "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": d2h_bytes,
                     "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": launches,
             "clocks": dict(clocks.summary(), kernel_sm_mhz=kernel_mhz,
                            kernel_sm_mhz_source="clock64 / globaltimer inside the last kernel of each operator"),
         }
-        if world == 1 and not args.no_sweep:
-            del hag, hrs
-            torch.cuda.empty_cache()
-            line["timing_protocol"] = timing_protocol_report(torch, api, {"ag_gemm": ag, "gemm_rs": rs})
+        if protocol is not None:
+            line["timing_protocol"] = protocol
             line["mlp_block"] = mlp_report(torch, api)
             torch.cuda.empty_cache()
-            line["interdecom"] = interdecom_report(torch, api, peaks["hbm_gbs"])
+            line["interdecom"] = interdecom_report(torch, api, peaks["hbm_gbs"], args.recalibrate)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w_ag, w_rs)
         print(json.dumps(line), flush=True)
@@ -662,6 +752,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the InterDecom sweep / calibration / selection report")
+    ap.add_argument("--recalibrate", action="store_true",
+                    help="fit the models' parameters in this run instead of loading the stored calibration")
     args = ap.parse_args()
     w_ag, w_rs = wl.C2_AG, wl.C3_RS
     if args.impl == "reference":

@@ -30,7 +30,7 @@
 // In the pair kernels each CTA loads its own rows of A and its half of the B
 // rows; the leader CTA issues tcgen05.mma.cta_group::2, which reads both CTAs'
 // shared memory, and each CTA's tensor memory receives its rows of the
-// accumulator.  No TMA load uses cluster multicast.
+// accumulator.  Every TMA load fills the shared memory of the CTA that issues it only.
 //
 // Warp roles (192 threads, 1 CTA per SM): warp 0 = TMA producer (one lane),
 // warp 1 = tensor-memory allocation + MMA issue (one lane), warps 2..5 =
@@ -86,9 +86,14 @@ struct Control {
   int abort;
 };
 
+// epilogue staging: per epilogue warp 32 rows x 64 BF16 columns, rows padded by 16 bytes (conflict-free 16-byte accesses)
+constexpr int kStageRowBytes = 64 * 2 + 16;
+constexpr int kStageWarpBytes = 32 * kStageRowBytes;
+
 template <bool kPair>
 constexpr size_t smem_bytes() {
-  return 1024 /*alignment slack*/ + size_t(Cfg<kPair>::kStages) * Cfg<kPair>::kStageBytes + sizeof(Control);
+  return 1024 /*alignment slack*/ + size_t(Cfg<kPair>::kStages) * Cfg<kPair>::kStageBytes + sizeof(Control) + 16 +
+         size_t(kEpilogueWarps) * kStageWarpBytes;
 }
 
 __device__ __forceinline__ void report_timeout(const GemmParams& p, Control* ctl, int site, int tile) {
@@ -469,24 +474,25 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
   } else {
     // ---------------------------------------------------------------- epilogue
     const int quarter = warp & 3;               // TMEM lanes this warp may touch
+    uint8_t* stage = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ctl + 1) + 15) & ~uintptr_t(15)) +
+                     (warp - 2) * kStageWarpBytes;
+    const int seg = lane & 7;                   // 16-byte segment of a 128-byte row piece this lane moves
     uint32_t it = 0;
     for (int t = unit; t < p.total_tiles; t += n_units, ++it) {
       const uint32_t buf = it & 1u;
       const uint32_t acc_phase = (it >> 1) & 1u;
-      if (!wait_bounded(&ctl->acc_full[buf], acc_phase, ctl, p, WAIT_ACC_FULL, t)) break;
-      tc_fence_after_sync();
       const TileCoord tc = decode_tile(p, t);
       const Frag frag = fragment_of(p, tc.blk, tc.mt * C::kTileRows + int(cta_rank) * BM);   // this CTA's 128 rows
       const BlockDesc& b = p.blocks[frag.blk];
-      const int row_in_block = frag.r0 + quarter * 32 + lane;
-      const bool row_ok = row_in_block < p.rows_per_block;
+      const int first_row = frag.r0 + quarter * 32;          // row (inside the block) of lane 0
       const int ncols = min(BN, p.N - tc.nt * BN);
-      const int nchunks = (ncols + 31) >> 5;
       // SwiGLU halves the columns: accumulator columns (2j, 2j+1) = (gate, up) give output column j
       const int act = kAct ? p.activation : int(ACT_NONE);
       const int oshift = act == ACT_SWIGLU ? 1 : 0;
-      __nv_bfloat16* orow = p.out[b.out_idx] + int64_t(b.out_row0 + row_in_block) * p.ldo + ((int64_t(tc.nt) * BN) >> oshift);
+      const int ocols = ncols >> oshift;
+      __nv_bfloat16* obase = p.out[b.out_idx] + int64_t(b.out_row0 + first_row) * p.ldo + ((int64_t(tc.nt) * BN) >> oshift);
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
+      const int npass = (ocols + 63) >> 6;
 
       // Ring read-modify-write: contributor `step` of a partition adds its
       // partial tile to the running sum that contributor step-1 left in the
@@ -497,85 +503,129 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       const bool rmw = p.epilogue == EPI_RING_RMW && frag.r0 < p.rows_per_block;   // a fragment past the block adds nothing
       const bool add_previous = rmw && b.step > 0;
       int* counter = nullptr;
+      // `sum` first holds this lane's row of the running sum (packed BF16 pairs), then the row to store.
+      uint32_t sum[BN / 2];
       if (rmw) {
         counter = p.tile_counters + (int64_t(b.part) * p.frags_m + frag.r0 / BM) * p.tiles_n + tc.nt;
         if (add_previous) {
+          // All of this happens while the tile's MMAs are still running: the wait for the previous
+          // contributor and the fetch of its running sum need nothing from the accumulator.
           int ready = 1;
           if (lane == 0) ready = wait_counter(counter, int(b.step) * kEpilogueWarps, ctl, p, t) ? 1 : 0;
           ready = __shfl_sync(0xffffffffu, ready, 0);
           // lane 0 acquired the counter; the warp barrier orders the other lanes' loads of the running sum behind it
           __syncwarp();
           if (!ready) break;
+          // The warp's 32 rows x 256 columns come in as whole 128-byte row pieces (4 rows per load instruction,
+          // every sector fully used), all 32 loads of a lane in flight at once, and are then transposed through
+          // shared memory, 64 columns at a time, into one row per lane (in place in `sum`).
+#pragma unroll
+          for (int pass = 0; pass < BN / 64; ++pass) {
+            const int col = pass * 64 + seg * 8;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int r = i * 4 + (lane >> 3);
+              uint4 piece = make_uint4(0u, 0u, 0u, 0u);
+              if (pass < npass && first_row + r < p.rows_per_block && col < ocols)
+                piece = __ldcg(reinterpret_cast<const uint4*>(obase + int64_t(r) * p.ldo + col));   // written by another SM: from L2
+              sum[pass * 32 + i * 4 + 0] = piece.x;
+              sum[pass * 32 + i * 4 + 1] = piece.y;
+              sum[pass * 32 + i * 4 + 2] = piece.z;
+              sum[pass * 32 + i * 4 + 3] = piece.w;
+            }
+          }
+#pragma unroll
+          for (int pass = 0; pass < BN / 64; ++pass) {
+            if (pass < npass) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                *reinterpret_cast<uint4*>(stage + (i * 4 + (lane >> 3)) * kStageRowBytes + seg * 16) =
+                    make_uint4(sum[pass * 32 + i * 4 + 0], sum[pass * 32 + i * 4 + 1], sum[pass * 32 + i * 4 + 2],
+                               sum[pass * 32 + i * 4 + 3]);
+              __syncwarp();
+#pragma unroll
+              for (int g = 0; g < 8; ++g) {
+                const uint4 q = *reinterpret_cast<const uint4*>(stage + lane * kStageRowBytes + g * 16);
+                sum[pass * 32 + g * 4 + 0] = q.x;
+                sum[pass * 32 + g * 4 + 1] = q.y;
+                sum[pass * 32 + g * 4 + 2] = q.z;
+                sum[pass * 32 + g * 4 + 3] = q.w;
+              }
+              __syncwarp();
+            }
+          }
         }
       }
-      // The running sum of this lane's row is fetched in one go, before the accumulator is read:
-      // the read-modify-write then pays one L2 round trip per tile instead of one per chunk.
-      uint4 prev[BN / 8];
-      if (add_previous && row_ok) {
-#pragma unroll
-        for (int g = 0; g < BN / 8; ++g)
-          if (g * 8 < ncols) prev[g] = __ldcg(reinterpret_cast<const uint4*>(orow + g * 8));   // written by another SM: from L2
-      }
+
+      if (!wait_bounded(&ctl->acc_full[buf], acc_phase, ctl, p, WAIT_ACC_FULL, t)) break;
+      tc_fence_after_sync();
+      // 1) accumulator row (256 columns) TMEM -> registers 32 columns at a time, running sum added in FP32,
+      //    packed to BF16 (sum[j] = output columns 2j, 2j+1)
 #pragma unroll
       for (int c = 0; c < BN / 32; ++c) {
-        if (c < nchunks) {
-          uint32_t v[32];
-          tmem_ld_32x32b_x32(taddr + c * 32, v);
-          tmem_ld_wait();
-          if (c == nchunks - 1) {
-            // accumulator fully copied to registers: hand it back to the MMA issuer
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) {
-              if (kPair) mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->acc_empty[buf]), 0));
-              else mbar_arrive(&ctl->acc_empty[buf]);
+        uint32_t v[32];
+        tmem_ld_32x32b_x32(taddr + c * 32, v);
+        tmem_ld_wait();
+        if (add_previous) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const uint32_t o = sum[c * 16 + i];
+            v[2 * i] = __float_as_uint(__uint_as_float(v[2 * i]) + __uint_as_float(o << 16));
+            v[2 * i + 1] = __float_as_uint(__uint_as_float(v[2 * i + 1]) + __uint_as_float(o & 0xFFFF0000u));
+          }
+        }
+        if (act == ACT_SWIGLU) {
+          // 32 accumulator columns -> 16 output columns, packed densely from register 0 on
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            sum[c * 8 + i] = pack_bf16x2(swiglu_f32(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1])),
+                                         swiglu_f32(__uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3])));
+        } else {
+          if (act == ACT_GELU_TANH) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(gelu_tanh_f32(__uint_as_float(v[i])));
+          }
+#pragma unroll
+          for (int i = 0; i < 16; ++i) sum[c * 16 + i] = pack_bf16x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+        }
+      }
+      // accumulator fully copied to registers: hand it back to the MMA issuer
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) {
+        if (kPair) mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->acc_empty[buf]), 0));
+        else mbar_arrive(&ctl->acc_empty[buf]);
+      }
+      // 2) registers -> padded shared memory -> global, 64 columns per pass: every store
+      //    instruction writes 4 rows x 128 contiguous bytes.
+#pragma unroll
+      for (int pass = 0; pass < BN / 64; ++pass) {
+        if (pass < npass) {
+          uint4* srow = reinterpret_cast<uint4*>(stage + lane * kStageRowBytes);
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            srow[g] = make_uint4(sum[pass * 32 + g * 4 + 0], sum[pass * 32 + g * 4 + 1], sum[pass * 32 + g * 4 + 2],
+                                 sum[pass * 32 + g * 4 + 3]);
+          __syncwarp();
+          const int col = pass * 64 + seg * 8;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int r = i * 4 + (lane >> 3);
+            if (first_row + r < p.rows_per_block && col < ocols) {
+              const uint4 q = *reinterpret_cast<const uint4*>(stage + r * kStageRowBytes + seg * 16);
+              *reinterpret_cast<uint4*>(obase + int64_t(r) * p.ldo + col) = q;
             }
           }
-          if (row_ok) {
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              if (c * 32 + g * 8 < ncols) {
-                float f[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[g * 8 + i]);
-                if (add_previous) {
-                  const uint4 o = prev[c * 4 + g];
-                  f[0] += __uint_as_float(o.x << 16);
-                  f[1] += __uint_as_float(o.x & 0xFFFF0000u);
-                  f[2] += __uint_as_float(o.y << 16);
-                  f[3] += __uint_as_float(o.y & 0xFFFF0000u);
-                  f[4] += __uint_as_float(o.z << 16);
-                  f[5] += __uint_as_float(o.z & 0xFFFF0000u);
-                  f[6] += __uint_as_float(o.w << 16);
-                  f[7] += __uint_as_float(o.w & 0xFFFF0000u);
-                }
-                if (act == ACT_SWIGLU) {
-                  uint2 h;
-                  h.x = pack_bf16x2(swiglu_f32(f[0], f[1]), swiglu_f32(f[2], f[3]));
-                  h.y = pack_bf16x2(swiglu_f32(f[4], f[5]), swiglu_f32(f[6], f[7]));
-                  *reinterpret_cast<uint2*>(orow + ((c * 32 + g * 8) >> 1)) = h;
-                } else {
-                  if (act == ACT_GELU_TANH) {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) f[i] = gelu_tanh_f32(f[i]);
-                  }
-                  uint4 q;
-                  q.x = pack_bf16x2(f[0], f[1]);
-                  q.y = pack_bf16x2(f[2], f[3]);
-                  q.z = pack_bf16x2(f[4], f[5]);
-                  q.w = pack_bf16x2(f[6], f[7]);
-                  *reinterpret_cast<uint4*>(orow + c * 32 + g * 8) = q;
-                }
-              }
-            }
-          }
+          __syncwarp();
         }
       }
       if (rmw) {
-        __threadfence();          // this lane's stores are visible device-wide before the counter moves
+        // The warp barrier orders every lane's stores before lane 0's release: the increment becomes visible
+        // device-wide only after the rows this warp wrote (release is cumulative over what the barrier ordered).
         __syncwarp();
         if (lane == 0) {
-          const int before = atomicAdd(counter, 1);
+          int before;
+          asm volatile("atom.add.release.gpu.global.s32 %0, [%1], 1;" : "=r"(before) : "l"(counter) : "memory");
           // the last warp of the last contributor leaves the counter at zero for the next call
           if (int(b.step) == p.last_step && before == (p.last_step + 1) * kEpilogueWarps - 1) atomicExch(counter, 0);
         }
@@ -616,9 +666,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 // 3 for small stages), which also holds across the change of kind.
 constexpr int kChunkBytes = BM * BK * 2;      // 16 KB: one 128-row, 64-column BF16 box
 constexpr int kChunks = 12;
-// epilogue staging: per epilogue warp 32 rows x 64 BF16 columns, rows padded by 16 bytes (conflict-free 16-byte accesses)
-constexpr int kStageRowBytes = 64 * 2 + 16;
-constexpr int kStageWarpBytes = 32 * kStageRowBytes;
 constexpr size_t kMixedSmemBytes =
     1024 + size_t(kChunks) * kChunkBytes + sizeof(Control) + 16 + size_t(kEpilogueWarps) * kStageWarpBytes;
 
@@ -988,7 +1035,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
       const MixedTile tile = decode_mixed(p, t);
       if (!tile.valid) continue;
       const int ncols = min(BN, p.N - tile.nt * BN);
-      const int nchunks = (ncols + 31) >> 5;
       const int n_acc = tile.big ? 2 : 1;
       for (int a = 0; a < n_acc && ok; ++a) {
         const uint32_t buf = tile.big ? uint32_t(a) : (small_rr & 1u);
@@ -1002,7 +1048,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
         const Frag frag = fragment_of(p, tile.blk, tile.row0 + (tile.big ? int(cta_rank) * 2 * BM + a * BM : int(cta_rank) * BM));
         const BlockDesc& b = p.blocks[frag.blk];
         const int row_in_block = frag.r0 + quarter * 32 + lane;
-        const bool row_ok = row_in_block < p.rows_per_block;
         // SwiGLU halves the columns: accumulator columns (2j, 2j+1) = (gate, up) give output column j
         const int act = kAct ? p.activation : int(ACT_NONE);
         const int oshift = act == ACT_SWIGLU ? 1 : 0;
