@@ -80,19 +80,23 @@ def measure_cases(cases, out_path, iters=5, log=print):
     stream = torch.cuda.current_stream()
     side = torch.cuda.Stream()
 
-    def median_ms(fn, iters, warm=1):
+    def timed_in_turn(fns, iters, warm=1):
+        """Median time of every variant, the variants timed in turn inside one loop: the board's power state drifts
+        while a case runs, and variants timed one after the other would not be compared at the same clock."""
         for _ in range(warm):
-            fn()
+            for fn in fns.values():
+                fn()
         torch.cuda.synchronize()
-        ts = []
+        ts = {k: [] for k in fns}
         for _ in range(iters):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            fn()
-            e1.record(stream)
-            torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1))
-        return float(np.median(ts))
+            for k, fn in fns.items():
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                fn()
+                e1.record(stream)
+                torch.cuda.synchronize()
+                ts[k].append(e0.elapsed_time(e1))
+        return {k: float(np.median(v)) for k, v in ts.items()}
 
     measured = 0
     for c in cases:
@@ -109,21 +113,25 @@ def measure_cases(cases, out_path, iters=5, log=print):
         ws = api.alloc_workspace(pr)
         fused = api.compass_ag_gemm if w.op == wl.OP_AG_GEMM else api.compass_gemm_rs
         rec = dict(c, flops=w.flops, m_rows=w.m)
-        rec["fused_ms"] = median_ms(lambda: fused(pr, A, B, out, ws, stream), iters)
+        fns = {"fused": lambda: fused(pr, A, B, out, ws, stream)}
+        pws = None
         if w.op == wl.OP_AG_GEMM:
             pws = torch.empty(api.compass_workspace_bytes(pr, api.WS_PUSH), dtype=torch.uint8, device="cuda")
             api.compass_workspace_init(pws)
-            rec["push_ms"] = median_ms(lambda: api.compass_ag_gemm_push(pr, A, B, out, pws, stream, side), iters)
-            del pws
+            fns["push"] = lambda: api.compass_ag_gemm_push(pr, A, B, out, pws, stream, side)
         dws = None
-        rec["decomp_ms"] = {}
         for d in DEGREES:
             if w.m % d:
                 continue
             prd = api.make_problem(w.op, w.P, w.M, w.N, w.K, d=d)
             if dws is None:
                 dws = api.alloc_workspace(prd, api.WS_DECOMP)
-            rec["decomp_ms"][str(d)] = median_ms(lambda: api.compass_decomp(prd, A, B, out, dws, stream, side), iters)
+            fns[str(d)] = (lambda prd: lambda: api.compass_decomp(prd, A, B, out, dws, stream, side))(prd)
+        ms = timed_in_turn(fns, iters)
+        rec["fused_ms"] = ms["fused"]
+        if "push" in ms:
+            rec["push_ms"] = ms["push"]
+        rec["decomp_ms"] = {k: v for k, v in ms.items() if k not in ("fused", "push")}
         status = api.compass_read_status(ws)
         if status != (api.OK, 0):
             raise SystemExit(f"device status {status} on {c}")
@@ -131,7 +139,7 @@ def measure_cases(cases, out_path, iters=5, log=print):
             f.write(json.dumps(rec) + "\n")
         log(case_key(c), round(rec["fused_ms"], 3), {k: round(v, 3) for k, v in rec["decomp_ms"].items()})
         measured += 1
-        del A, B, out, ws, dws
+        del A, B, out, ws, dws, pws, fns
         torch.cuda.empty_cache()
     return measured
 
