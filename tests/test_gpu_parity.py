@@ -104,6 +104,47 @@ def test_tensor_map_cache_serves_repeats_and_misses_on_new_buffers_or_shapes():
     assert api.tensor_map_cache_stats()[1] > m2
 
 
+def test_two_host_threads_call_the_library_concurrently():
+    """The launch descriptors and the tensor-map table are per host thread and the per-device facts are behind a
+    mutex: two threads, each with its own stream, workspace and buffers, call the fused operators at the same time
+    (the kernels used here wait on nothing outside their own CTA pair, so they may share the GPU)."""
+    import threading
+
+    cases = [small(wl.OP_AG_GEMM, 4, 512, 520, 200, seed=3, dist=0.1), small(wl.OP_GEMM_RS, 4, 512, 264, 328, seed=4, dist=0.05)]
+    inputs = [wl.make_inputs(w) for w in cases]
+    refs = [ops.ag_gemm(*inputs[0]), ops.gemm_rs(*inputs[1])]
+    results, errors = [None, None], []
+
+    def worker(i):
+        try:
+            w = cases[i]
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                A, B = gu.device_inputs(*inputs[i])
+                pr = gu.problem_of(w)
+                ws = api.alloc_workspace(pr)
+                outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+                stream.synchronize()
+                call = api.compass_ag_gemm if w.op == wl.OP_AG_GEMM else api.compass_gemm_rs
+                for _ in range(25):
+                    call(pr, A, B, [o.view for o in outs], ws, stream)
+                assert api.compass_read_status(ws, stream) == (api.OK, 0)
+                stream.synchronize()
+                assert all(o.guards_intact() for o in outs)
+                results[i] = [o.bits() for o in outs]
+        except Exception as e:      # surfaces in the main thread
+            errors.append((i, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for i in range(2):
+        check_all(results[i], refs[i], cases[i].name)
+
+
 def test_config1_ag_gemm_full():
     w = wl.C1_AG
     A, B = wl.make_inputs(w)
