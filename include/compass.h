@@ -254,6 +254,19 @@ int compass_decomp(const compass_problem* problem, const void* const* A, const v
                    void* const* out, void* workspace, size_t workspace_bytes,
                    void* stream_compute, void* stream_copy);
 
+/* The d sub-collectives of compass_decomp alone, without the sub-GEMMs: what
+ * Section IV-C calls T_comm, made measurable on its own (the sub-AllGathers
+ * of AG: every shard's row slices into the P gather buffers; the
+ * sub-ReduceScatters of RS: the P BF16 partial buffers of the workspace, as
+ * they are -- zero after compass_workspace_init, or what the last
+ * compass_decomp left there -- summed into `out`).  Same arguments, streams
+ * and ordering as compass_decomp; B is not read.  These phases are bound by
+ * HBM bandwidth: AG reads M*K*2 bytes and writes P times that, RS reads
+ * P*M*N*2 bytes and writes M*N*2. */
+int compass_decomp_comm(const compass_problem* problem, const void* const* A, const void* const* B,
+                        void* const* out, void* workspace, size_t workspace_bytes,
+                        void* stream_compute, void* stream_copy);
+
 /* ---- strategy selector (Algorithm 1, Eq. 2-8) ------------------------------
  * T_comp, T_comm and lambda come from the calibrated linear models; the
  * decomposition degree d* from Eq. 4-5 (restricted to degrees that divide

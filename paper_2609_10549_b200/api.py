@@ -38,7 +38,7 @@ EXPORTS = (
     "compass_read_status", "compass_launch_plan", "compass_fused_host", "compass_status_string",
     "compass_last_cuda_error", "compass_kernel_launch_count", "compass_gemm_rs_sequential_noalloc",
     "compass_set_wait_limit_us", "compass_calib_fit_line", "compass_ag_gemm_push", "compass_read_kernel_clock",
-    "compass_mlp_workspace_bytes", "compass_mlp_block", "compass_noalloc_read_status", "compass_select_ex", "compass_test_drop_flag_writes", "compass_tensor_map_cache_stats",
+    "compass_mlp_workspace_bytes", "compass_mlp_block", "compass_noalloc_read_status", "compass_select_ex", "compass_test_drop_flag_writes", "compass_tensor_map_cache_stats", "compass_decomp_comm",
 )
 
 
@@ -95,6 +95,7 @@ def lib() -> C.CDLL:
         for name in ("compass_ag_gemm", "compass_gemm_rs"):
             getattr(L, name).argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p]
         L.compass_decomp.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.compass_decomp_comm.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.compass_ag_gemm_push.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.compass_mlp_workspace_bytes.argtypes = [C.POINTER(Mlp), C.POINTER(C.c_size_t)]
         L.compass_mlp_block.argtypes = [C.POINTER(Mlp), pp, pp, pp, pp, pp, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -343,6 +344,16 @@ def compass_decomp(problem: Problem, A: Sequence, B: Sequence, out: Sequence, wo
     sp = _stream_handle(stream_copy) if stream_copy is not None else sc
     _check(lib().compass_decomp(C.byref(problem), _ptr_array(A), _ptr_array(B), _ptr_array(out), p, n, sc, sp),
            "compass_decomp")
+
+
+def compass_decomp_comm(problem: Problem, A: Sequence, B: Sequence, out: Sequence, workspace, stream_compute=None,
+                        stream_copy=None) -> None:
+    """The d sub-collectives of compass_decomp alone (no sub-GEMMs): T_comm, measurable on its own."""
+    p, n = _ws(workspace)
+    sc = _stream_handle(stream_compute)
+    sp = _stream_handle(stream_copy) if stream_copy is not None else sc
+    _check(lib().compass_decomp_comm(C.byref(problem), _ptr_array(A), _ptr_array(B), _ptr_array(out), p, n, sc, sp),
+           "compass_decomp_comm")
 
 
 def compass_gemm_rs_sequential_noalloc(problem: Problem, A: Sequence, B: Sequence, Out: Sequence, stream=None) -> None:

@@ -319,8 +319,9 @@ struct EventPool {
 };
 EventPool g_events;
 
+// comm_only: enqueue the sub-collectives alone (the T_comm of Section IV-C), without the sub-GEMMs.
 int decomp_ag(const compass_problem* pr, const void* const* A, const void* const* B, void* const* C, uint8_t* ws,
-              cudaStream_t s_comp, cudaStream_t s_copy, cudaEvent_t* ev) {
+              cudaStream_t s_comp, cudaStream_t s_copy, cudaEvent_t* ev, bool comm_only) {
   const int P = pr->P, d = pr->d;
   const int64_t m = pr->M / P, K = pr->K, sl = m / d;
   const size_t gather_bytes = align_up(size_t(pr->M) * size_t(K) * 2);
@@ -367,6 +368,7 @@ int decomp_ag(const compass_problem* pr, const void* const* A, const void* const
     }
     if ((e = cudaEventRecord(ev[1 + j], s_copy)) != cudaSuccess) return record_cuda_error(e);
     if ((e = cudaStreamWaitEvent(s_comp, ev[1 + j], 0)) != cudaSuccess) return record_cuda_error(e);
+    if (comm_only) continue;
     // sub-GEMM j on the gathered rows
     // rank-major, like the fused launch: a rank's weight shard stays in L2 across its P row slices
     int n = 0;
@@ -388,7 +390,7 @@ int decomp_ag(const compass_problem* pr, const void* const* A, const void* const
 }
 
 int decomp_rs(const compass_problem* pr, const void* const* A, const void* const* B, void* const* Out, uint8_t* ws,
-              cudaStream_t s_comp, cudaStream_t s_copy, cudaEvent_t* ev) {
+              cudaStream_t s_comp, cudaStream_t s_copy, cudaEvent_t* ev, bool comm_only) {
   const int P = pr->P, d = pr->d;
   const int64_t m = pr->M / P, sl = m / d;
   const size_t partial_bytes = align_up(size_t(pr->M) * size_t(pr->N) * 2);
@@ -429,7 +431,7 @@ int decomp_rs(const compass_problem* pr, const void* const* A, const void* const
         b.out_row0 = b.a_row0;
       }
     L.n_blocks = n;
-    int st = launch_gemm(L, s_comp);
+    int st = comm_only ? int(COMPASS_OK) : launch_gemm(L, s_comp);
     if (st != COMPASS_OK) return st;
     if ((e = cudaEventRecord(ev[1 + j], s_comp)) != cudaSuccess) return record_cuda_error(e);
     if ((e = cudaStreamWaitEvent(s_copy, ev[1 + j], 0)) != cudaSuccess) return record_cuda_error(e);
@@ -735,8 +737,8 @@ extern "C" int compass_ag_gemm_push(const compass_problem* pr, const void* const
   return COMPASS_OK;
 }
 
-extern "C" int compass_decomp(const compass_problem* pr, const void* const* A, const void* const* B, void* const* out,
-                              void* ws, size_t ws_bytes, void* stream_compute, void* stream_copy) {
+static int decomp_call(const compass_problem* pr, const void* const* A, const void* const* B, void* const* out, void* ws,
+                       size_t ws_bytes, void* stream_compute, void* stream_copy, bool comm_only) {
   int st = validate_problem(pr, -1, true);
   if (st != COMPASS_OK) return st;
   if (pr->d > 16) return COMPASS_ERR_UNSUPPORTED;
@@ -748,8 +750,18 @@ extern "C" int compass_decomp(const compass_problem* pr, const void* const* A, c
   st = g_events.ensure(pr->d + 1);
   if (st != COMPASS_OK) return st;
   cudaStream_t sc = static_cast<cudaStream_t>(stream_compute), sp = static_cast<cudaStream_t>(stream_copy);
-  if (pr->op == COMPASS_OP_AG_GEMM) return decomp_ag(pr, A, B, out, static_cast<uint8_t*>(ws), sc, sp, g_events.ev);
-  return decomp_rs(pr, A, B, out, static_cast<uint8_t*>(ws), sc, sp, g_events.ev);
+  if (pr->op == COMPASS_OP_AG_GEMM) return decomp_ag(pr, A, B, out, static_cast<uint8_t*>(ws), sc, sp, g_events.ev, comm_only);
+  return decomp_rs(pr, A, B, out, static_cast<uint8_t*>(ws), sc, sp, g_events.ev, comm_only);
+}
+
+extern "C" int compass_decomp(const compass_problem* pr, const void* const* A, const void* const* B, void* const* out,
+                              void* ws, size_t ws_bytes, void* stream_compute, void* stream_copy) {
+  return decomp_call(pr, A, B, out, ws, ws_bytes, stream_compute, stream_copy, false);
+}
+
+extern "C" int compass_decomp_comm(const compass_problem* pr, const void* const* A, const void* const* B, void* const* out,
+                                   void* ws, size_t ws_bytes, void* stream_compute, void* stream_copy) {
+  return decomp_call(pr, A, B, out, ws, ws_bytes, stream_compute, stream_copy, true);
 }
 
 extern "C" int compass_fused_host(const compass_problem* pr, const void* const* A_host, const void* const* B_host,

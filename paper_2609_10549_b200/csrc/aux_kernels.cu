@@ -81,12 +81,29 @@ struct GatherParams {
 __global__ void __launch_bounds__(256) gather_slices_kernel(const __grid_constant__ GatherParams p) {
   const int64_t per_shard = p.slice_rows * p.k_vec;
   const int64_t total = per_shard * p.P;
-  for (int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += int64_t(gridDim.x) * blockDim.x) {
-    const int q = int(i / per_shard);
-    const int64_t w = i - int64_t(q) * per_shard;
-    const uint4 v = __ldg(p.shard[q] + p.slice_begin * p.k_vec + w);
-    const int64_t dst = (int64_t(q) * p.m + p.slice_begin) * p.k_vec + w;
-    for (int r = 0; r < p.P; ++r) p.gather[r][dst] = v;
+  const int64_t stride = int64_t(gridDim.x) * blockDim.x;
+  // Four vectors per thread are fetched before the first is stored (64 bytes of reads in flight per thread); every
+  // vector then goes to the P gather buffers with streaming stores: the copies are not read again by this kernel and
+  // should not push the GEMM's operands out of L2.
+  constexpr int kUnroll = 4;
+  for (int64_t i0 = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i0 < total; i0 += stride * kUnroll) {
+    uint4 v[kUnroll];
+    int64_t dst[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int64_t i = i0 + u * stride;
+      dst[u] = -1;
+      if (i < total) {
+        const int q = int(i / per_shard);
+        const int64_t w = i - int64_t(q) * per_shard;
+        v[u] = __ldg(p.shard[q] + p.slice_begin * p.k_vec + w);
+        dst[u] = (int64_t(q) * p.m + p.slice_begin) * p.k_vec + w;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u)
+      if (dst[u] >= 0)
+        for (int r = 0; r < p.P; ++r) __stcs(p.gather[r] + dst[u], v[u]);
   }
 }
 

@@ -5,8 +5,9 @@
     python -m paper_2609_10549_b200.run_case --op ag --variant decomp --d 4 --P 4 --M 4096 --N 3072 --K 4096
 
 --op ag|rs: AllGather+GEMM (N per rank, K full) or GEMM+ReduceScatter (K per rank, N full).
---variant fused|ring|push|decomp: the fused kernel (gather by address / segmented K), the ring
-read-modify-write GEMM+ReduceScatter, the readiness-driven AllGather+GEMM, or InterDecom with --d stages.
+--variant fused|ring|push|decomp|comm: the fused kernel (gather by address / segmented K), the ring
+read-modify-write GEMM+ReduceScatter, the readiness-driven AllGather+GEMM, InterDecom with --d stages, or the --d
+sub-collectives of InterDecom alone (gather / reduce kernels on one stream; reported in GB/s of their algorithmic bytes).
 Inputs are drawn on the device (seeded); every launch is timed between its own pair of CUDA events on the
 launching stream after --warmup untimed launches.  Prints one JSON line: median / best milliseconds,
 TFLOP/s over the FLOPs of all P logical ranks, the host time of one call, and the SM clock the last kernel
@@ -24,7 +25,7 @@ import numpy as np
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--op", choices=["ag", "rs"], required=True)
-    ap.add_argument("--variant", choices=["fused", "ring", "push", "decomp"], default="fused")
+    ap.add_argument("--variant", choices=["fused", "ring", "push", "decomp", "comm"], default="fused")
     ap.add_argument("--P", type=int, required=True)
     ap.add_argument("--M", type=int, required=True)
     ap.add_argument("--N", type=int, required=True)
@@ -71,6 +72,9 @@ def main():
     elif args.variant == "push":
         ws = api.alloc_workspace(pr, api.WS_PUSH)
         run = lambda: api.compass_ag_gemm_push(pr, A, B, out, ws, stream, side)
+    elif args.variant == "comm":
+        ws = api.alloc_workspace(pr, api.WS_DECOMP)
+        run = lambda: api.compass_decomp_comm(pr, A, B, out, ws, stream, None)
     else:
         ws = api.alloc_workspace(pr, api.WS_DECOMP)
         run = lambda: api.compass_decomp(pr, A, B, out, ws, stream, side)
@@ -92,6 +96,13 @@ def main():
         raise SystemExit(f"device-side status {status}")
     cycles, ns = api.compass_read_kernel_clock(ws)
     med = float(np.median(ts))
+    if args.variant == "comm":
+        # AllGather: every shard read once, written to the P gather buffers; ReduceScatter: P partials read, one result written
+        nbytes = 2.0 * w.M * w.K * (1 + w.P) if op == wl.OP_AG_GEMM else 2.0 * w.M * w.N * (w.P + 1)
+        print(json.dumps({"op": args.op, "variant": "comm", "P": w.P, "M": w.M, "N": w.N, "K": w.K, "d": args.d,
+                          "ms_median": med, "ms_best": float(np.min(ts)), "algorithmic_bytes": nbytes,
+                          "gbs_median": nbytes / (med * 1e-3) / 1e9}), flush=True)
+        return
     print(json.dumps({
         "op": args.op, "variant": args.variant, "P": w.P, "M": w.M, "N": w.N, "K": w.K, "d": args.d, "rings": args.rings,
         "order": args.order, "layout": args.layout, "iters": args.iters,

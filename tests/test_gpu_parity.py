@@ -404,6 +404,50 @@ def test_config4_interdecom_every_element(w, d):
     check_every_element(w, outs, f"{w.name} d={d}", one_rounding=w.op == wl.OP_AG_GEMM)
 
 
+def test_interdecom_collectives_alone():
+    """compass_decomp_comm runs the sub-collectives of InterDecom without the sub-GEMMs.  AllGather: afterwards every
+    rank's gather buffer in the workspace holds the concatenation of all shards, bit for bit.  ReduceScatter: on the
+    partial products a full compass_decomp left in the workspace it reproduces that call's output, bit for bit, for any d."""
+    w = small(wl.OP_AG_GEMM, 4, 512, 264, 200, dist=0.1)
+    A_bits, B_bits = wl.make_inputs(w)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    side = torch.cuda.Stream()
+    for d in (1, 4):
+        pr = gu.problem_of(w, d=d)
+        ws = api.alloc_workspace(pr, api.WS_DECOMP)
+        ws[api.STATUS_BYTES:].fill_(0x5A)
+        outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        api.compass_decomp_comm(pr, A, B, [o.view for o in outs], ws, torch.cuda.current_stream(), side)
+        assert api.compass_read_status(ws) == (api.OK, 0)
+        torch.cuda.synchronize()
+        gathered = np.concatenate(A_bits)
+        per_rank = (ws.numel() - api.STATUS_BYTES) // w.P
+        for r in range(w.P):
+            buf = ws[api.STATUS_BYTES + r * per_rank:api.STATUS_BYTES + r * per_rank + gathered.size * 2]
+            assert np.array_equal(buf.view(torch.int16).cpu().numpy().view(np.uint16).reshape(gathered.shape), gathered)
+        assert all(bool((o.full[gu.GUARD_ROWS:gu.GUARD_ROWS + o.rows] == gu.NAN_BITS).all()) for o in outs)   # no GEMM ran
+
+    w = small(wl.OP_GEMM_RS, 4, 512, 264, 200, dist=0.05)
+    A_bits, B_bits = wl.make_inputs(w)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    pr = gu.problem_of(w, d=1)
+    ws = api.alloc_workspace(pr, api.WS_DECOMP)
+    full = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    api.compass_decomp(pr, A, B, [o.view for o in full], ws, torch.cuda.current_stream(), side)
+    torch.cuda.synchronize()
+    launches = api.kernel_launch_count()
+    for d in (1, 8):
+        again = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        api.compass_decomp_comm(gu.problem_of(w, d=d), A, B, [o.view for o in again], ws, torch.cuda.current_stream(), side)
+        assert api.compass_read_status(ws) == (api.OK, 0)
+        torch.cuda.synchronize()
+        assert all(o.guards_intact() for o in again)
+        for x, y in zip(full, again):
+            assert np.array_equal(x.bits(), y.bits())
+    assert api.kernel_launch_count() == launches + 1 + 8            # reduce kernels only
+    check_all([o.bits() for o in full], ops.gemm_rs(A_bits, B_bits), w.name)
+
+
 @pytest.mark.parametrize("op", [wl.OP_AG_GEMM, wl.OP_GEMM_RS])
 def test_host_buffer_entry_point(op):
     w = small(op, 2, 256, 264, 200, dist=0.1)
