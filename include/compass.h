@@ -427,7 +427,7 @@ int compass_set_wait_limit_us(uint32_t microseconds);
 /* The library keeps the TMA tensor maps it encodes in a small per-thread
  * table keyed by (base pointer, rows, row length, box): repeated calls on the
  * same buffers skip the driver's encoding call (about a microsecond per map,
- * 3P maps per fused launch).  A map describes addresses and shapes, not
+ * 2P maps per fused launch).  A map describes addresses and shapes, not
  * contents, so the table never needs invalidating; a changed pointer or shape
  * is a new key.  This call reports, over all threads since the library was
  * loaded, how many map requests were served from the table and how many were

@@ -1168,20 +1168,21 @@ bool encode_kmajor_uncached(CUtensorMap* map, const void* ptr, int64_t rows, int
   return r == CUDA_SUCCESS;
 }
 
-// Encoded tensor maps are kept per host thread in a small direct-mapped table keyed by everything the
+// Encoded tensor maps are kept per host thread in a small 4-way set-associative table keyed by everything the
 // encoding depends on (base pointer, rows, row length, box rows): a training loop calls the same operator
-// on the same buffers over and over, and the driver call costs about a microsecond per map (3P maps per
+// on the same buffers over and over, and the driver call costs about a microsecond per map (2P maps per
 // fused launch, d times that for InterDecom).  A map describes addresses and shapes, not contents, so an
 // entry never goes stale; a different pointer or shape is a different key and is encoded afresh.
 struct MapCache {
-  static constexpr int kEntries = 256;
+  static constexpr int kSets = 64, kWays = 4;
   struct Key {
     const void* ptr;
     int64_t rows, cols;
     int32_t box_rows, valid;
   };
-  Key key[kEntries] = {};
-  alignas(64) CUtensorMap map[kEntries];
+  Key key[kSets][kWays] = {};
+  uint8_t next_way[kSets] = {};          // round-robin replacement inside a set
+  alignas(64) CUtensorMap map[kSets][kWays];
 };
 std::atomic<uint64_t> g_map_hits{0}, g_map_misses{0};
 
@@ -1190,14 +1191,24 @@ bool encode_kmajor(CUtensorMap* map, const void* ptr, int64_t rows, int64_t K, i
   uint64_t h = uint64_t(reinterpret_cast<uintptr_t>(ptr)) >> 4;
   h = (h ^ (h >> 17) ^ (uint64_t(rows) * 0x9E3779B97F4A7C15ull) ^ (uint64_t(K) * 0xC2B2AE3D27D4EB4Full) ^ uint64_t(box_rows)) *
       0xD6E8FEB86659FD93ull;
-  const int slot = int(h >> 56) & (MapCache::kEntries - 1);
-  MapCache::Key& k = cache.key[slot];
-  if (k.valid && k.ptr == ptr && k.rows == rows && k.cols == K && k.box_rows == box_rows) {
-    *map = cache.map[slot];
-    g_map_hits.fetch_add(1, std::memory_order_relaxed);
-    return true;
+  const int set = int(h >> 58) & (MapCache::kSets - 1);
+  for (int w = 0; w < MapCache::kWays; ++w) {
+    const MapCache::Key& k = cache.key[set][w];
+    if (k.valid && k.ptr == ptr && k.rows == rows && k.cols == K && k.box_rows == box_rows) {
+      *map = cache.map[set][w];
+      g_map_hits.fetch_add(1, std::memory_order_relaxed);
+      return true;
+    }
   }
-  if (!encode_kmajor_uncached(&cache.map[slot], ptr, rows, K, box_rows)) {
+  int way = -1;
+  for (int w = 0; w < MapCache::kWays && way < 0; ++w)
+    if (!cache.key[set][w].valid) way = w;
+  if (way < 0) {
+    way = cache.next_way[set];
+    cache.next_way[set] = uint8_t((way + 1) % MapCache::kWays);
+  }
+  MapCache::Key& k = cache.key[set][way];
+  if (!encode_kmajor_uncached(&cache.map[set][way], ptr, rows, K, box_rows)) {
     k.valid = 0;
     return false;
   }
@@ -1206,7 +1217,7 @@ bool encode_kmajor(CUtensorMap* map, const void* ptr, int64_t rows, int64_t K, i
   k.cols = K;
   k.box_rows = box_rows;
   k.valid = 1;
-  *map = cache.map[slot];
+  *map = cache.map[set][way];
   g_map_misses.fetch_add(1, std::memory_order_relaxed);
   return true;
 }
