@@ -145,6 +145,32 @@ def test_two_host_threads_call_the_library_concurrently():
         check_all(results[i], refs[i], cases[i].name)
 
 
+@pytest.mark.parametrize("variant", ["push", "decomp-1", "decomp-2", "decomp-4", "decomp-8", "decomp-16", "single-ring", "step-major"])
+def test_config1_variants(variant):
+    """Configuration 1 (P = 2, 128-row partitions) through every other path, every element against the oracle."""
+    w = wl.C1_AG
+    A, B = wl.make_inputs(w)
+    ref = ops.ag_gemm(A, B)
+    if variant == "push":
+        (outs,) = run_push(w, A, B)
+    elif variant.startswith("decomp"):
+        outs, status, guards = gu.run_decomp(w, A, B, int(variant.split("-")[1]))
+        assert status == (api.OK, 0) and guards
+    elif variant == "single-ring":
+        outs, status, guards = gu.run_fused(w, A, B, rings=1)
+        assert status == (api.OK, 0) and guards
+        assert np.array_equal(api.compass_schedule(w.op, w.P, 1, w.M), oracle_schedule(w.op, w.P, 1, w.M))
+    else:
+        pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, order=api.ORDER_STEP_MAJOR)
+        dA, dB = gu.device_inputs(A, B)
+        g = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        ws = api.alloc_workspace(pr)
+        api.compass_ag_gemm(pr, dA, dB, [o.view for o in g], ws)
+        assert api.compass_read_status(ws) == (api.OK, 0) and all(o.guards_intact() for o in g)
+        outs = [o.bits() for o in g]
+    check_all(outs, ref, f"{w.name} {variant}")
+
+
 def test_config1_ag_gemm_full():
     w = wl.C1_AG
     A, B = wl.make_inputs(w)
@@ -328,26 +354,34 @@ def _reference(w, idx, cache):
 
 
 def check_every_element(w, outs, what, ring_rmw=False, one_rounding=True, cache=True, block_rows=2048):
-    """All elements of all P outputs against the oracle.  The comparison runs over row blocks (its FP64
-    temporaries stay small) with max|ref| taken over the rank's whole tensor, as the acceptance rule says."""
-    rms_limit = 2.0 ** -9 * max(1.0, w.P ** 0.5) if ring_rmw else compare.RMS_REL_LIMIT
+    """All elements of all P outputs against the oracle (one variant; see check_variants_every_element)."""
+    check_variants_every_element(w, {what: (outs, ring_rmw, one_rounding)}, cache=cache, block_rows=block_rows)
+
+
+def check_variants_every_element(w, variants, cache=True, block_rows=2048):
+    """variants: {name: (outs, ring_rmw, one_rounding)}.  All elements of all P outputs of every variant against
+    the oracle; the FP64 reference of a rank / owner chunk is computed once and serves all variants.  The comparison
+    runs over row blocks (its FP64 temporaries stay small) with max|ref| taken over the rank's whole tensor, as the
+    acceptance rule says."""
     for r in range(w.P):
         ref = _reference(w, r, cache)
-        assert outs[r].shape == ref.shape
         max_ref = float(np.max(np.abs(ref)))
-        within, n = 0.0, 0
-        for lo in range(0, ref.shape[0], block_rows):
-            rep = compare.check(outs[r][lo:lo + block_rows], ref[lo:lo + block_rows], max_ref=max_ref)
-            assert rep.violations == 0 and rep.rms_rel <= rms_limit, f"{what} rank/chunk {r} rows {lo}+: {rep}"
-            rows = ref[lo:lo + block_rows].shape[0]
-            within += rep.frac_within_1ulp * rows
-            n += rows
-        # FP32 accumulation and one rounding: almost every element is the correctly rounded BF16 or its neighbour.
-        # The exceptions are results that nearly cancel: the FP32 sum of K terms carries an absolute error of about
-        # sqrt(K) * 2^-24 of the typical magnitude, which exceeds a BF16 step only for elements below ~2^-9 of it
-        # (a fraction of about 0.1 % at K = 28672, the longest contraction here).
-        if one_rounding and not ring_rmw:
-            assert within / n > 0.997, f"{what} rank/chunk {r}: only {within / n:.5f} of the elements within one BF16 step"
+        for what, (outs, ring_rmw, one_rounding) in variants.items():
+            rms_limit = 2.0 ** -9 * max(1.0, w.P ** 0.5) if ring_rmw else compare.RMS_REL_LIMIT
+            assert outs[r].shape == ref.shape
+            within, n = 0.0, 0
+            for lo in range(0, ref.shape[0], block_rows):
+                rep = compare.check(outs[r][lo:lo + block_rows], ref[lo:lo + block_rows], max_ref=max_ref)
+                assert rep.violations == 0 and rep.rms_rel <= rms_limit, f"{what} rank/chunk {r} rows {lo}+: {rep}"
+                rows = ref[lo:lo + block_rows].shape[0]
+                within += rep.frac_within_1ulp * rows
+                n += rows
+            # FP32 accumulation and one rounding: almost every element is the correctly rounded BF16 or its neighbour.
+            # The exceptions are results that nearly cancel: the FP32 sum of K terms carries an absolute error of about
+            # sqrt(K) * 2^-24 of the typical magnitude, which exceeds a BF16 step only for elements below ~2^-9 of it
+            # (a fraction of about 0.1 % at K = 28672, the longest contraction here).
+            if one_rounding and not ring_rmw:
+                assert within / n > 0.997, f"{what} rank/chunk {r}: only {within / n:.5f} of the elements within one BF16 step"
         del ref
 
 
@@ -366,14 +400,58 @@ def test_fused_every_element(w):
     check_every_element(w, outs, w.name)
 
 
-@pytest.mark.parametrize("w", [wl.C5_AG, wl.C5_RS], ids=lambda w: w.name)
-def test_config5_fused_every_element(w):
-    """The 70B-class pair: 1.5e13 and 7.7e12 FLOP of FP64 reference, one rank / owner chunk at a time."""
-    A, B = _inputs(w)
-    outs, status, guards = gu.run_fused(w, A, B)
-    assert status == (api.OK, 0) and guards
+def test_config5_ag_gemm_every_element_all_variants():
+    """The 70B-class AllGather+GEMM (1.5e13 FLOP of FP64 reference, one rank at a time): the fused kernel against the
+    oracle, every element; the push variant and InterDecom (d = 4) must reproduce the fused kernel's bits (they sum
+    every element over k in the same order), which is compared on the device."""
+    w = wl.C5_AG
+    A_bits, B_bits = _inputs(w)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    pr = gu.problem_of(w)
+    fused = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    ws = api.alloc_workspace(pr)
+    api.compass_ag_gemm(pr, A, B, [o.view for o in fused], ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    side = torch.cuda.Stream()
+    for name in ("push", "decomp d=4"):
+        other = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        if name == "push":
+            ws2 = api.alloc_workspace(pr, api.WS_PUSH)
+            api.compass_ag_gemm_push(pr, A, B, [o.view for o in other], ws2, torch.cuda.current_stream(), side)
+        else:
+            prd = gu.problem_of(w, d=4)
+            ws2 = api.alloc_workspace(prd, api.WS_DECOMP)
+            api.compass_decomp(prd, A, B, [o.view for o in other], ws2, torch.cuda.current_stream(), side)
+        assert api.compass_read_status(ws2) == (api.OK, 0)
+        torch.cuda.synchronize()
+        for r in range(w.P):
+            assert torch.equal(other[r].full, fused[r].full), f"{name}: rank {r} differs from the fused kernel (or wrote a guard row)"
+        del other, ws2
+        torch.cuda.empty_cache()
+    assert all(o.guards_intact() for o in fused)
+    outs = [o.bits() for o in fused]
+    del fused, A, B
+    torch.cuda.empty_cache()
     try:
         check_every_element(w, outs, w.name, cache=False)
+    finally:
+        _drop_cached(w)
+
+
+def test_config5_gemm_rs_every_element_all_variants():
+    """The 70B-class GEMM+ReduceScatter (7.7e12 FLOP of FP64 reference, one owner chunk at a time, computed once for
+    the three variants): segmented K, ring read-modify-write and InterDecom (d = 4), every element of each."""
+    w = wl.C5_RS
+    A, B = _inputs(w)
+    seg, status, guards = gu.run_fused(w, A, B)
+    assert status == (api.OK, 0) and guards
+    ring, status, guards = gu.run_fused(w, A, B, rs_variant=api.RS_RING_RMW)
+    assert status == (api.OK, 0) and guards
+    dec, status, guards = gu.run_decomp(w, A, B, 4)
+    assert status == (api.OK, 0) and guards
+    try:
+        check_variants_every_element(w, {f"{w.name} segmented-K": (seg, False, True), f"{w.name} ring-RMW": (ring, True, False),
+                                         f"{w.name} InterDecom d=4": (dec, False, False)}, cache=False)
     finally:
         _drop_cached(w)
 
