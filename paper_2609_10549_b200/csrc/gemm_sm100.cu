@@ -16,8 +16,8 @@
 // Three kernels share the roles and the barrier protocol:
 //   gemm_mixed_kernel  clusters of two CTAs; 512x256 tiles (two accumulators per
 //                      CTA sharing one B tile) for the whole waves of a launch,
-//                      256x256 tiles for the tail; plain-store epilogue.  The
-//                      default for blocks of >= 256 rows.
+//                      256x256 and 256x128 tiles for the tail; plain-store
+//                      epilogue.  The default wherever CTA pairs can be used.
 //   gemm_kernel<true>  clusters of two CTAs, 256x256 tiles; carries the ring
 //                      read-modify-write epilogue.
 //   gemm_kernel<false> one CTA per 128x256 tile; row fragments below 256 rows.
@@ -36,6 +36,7 @@
 // warp 1 = tensor-memory allocation + MMA issue (one lane), warps 2..5 =
 // epilogue (warp w reads TMEM lanes 32*(w%4)..+31).  Every wait is bounded and
 // reports COMPASS_ERR_TIMEOUT instead of hanging.
+#include <algorithm>
 #include <atomic>
 #include <mutex>
 
@@ -650,43 +651,60 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 
 // ---- mixed-tile pair kernel ---------------------------------------------------------
 //
-// Same roles and protocol as gemm_kernel<true>, but a launch holds two kinds of
-// tiles, both computed by a pair of CTAs:
+// Same roles and protocol as gemm_kernel<true>, but a launch holds up to three kinds
+// of tiles, all computed by a pair of CTAs:
 //   big   512 x 256: each CTA owns 256 rows as two 128-row accumulators (TMEM
 //         columns 0..255 and 256..511) that share one B tile.  A k-stage is one
 //         64-wide atom: A block 0, A block 1, B = 3 chunks of 16 KB per CTA,
 //         8 MMAs.  Per 128x256x64 MMA block the CTA loads 24 KB instead of 32.
 //   small 256 x 256: one accumulator, k-stage = two 64-wide atoms (A0, A1, B0,
 //         B1 = 4 chunks), 8 MMAs; accumulators alternate so the epilogue overlaps.
+//   quarter 256 x 128: one 128-column accumulator, k-stage = two atoms of A and
+//         this CTA's 64 B rows of both atoms in one chunk (3 chunks), 8 MMAs of
+//         half the width; bound by operand delivery, used only where it lets
+//         the last round over the pairs end sooner.
 // Big tiles come first and fill whole waves (their number is a multiple of the
-// number of pairs); the remaining rows are cut into small tiles so that the last,
-// partly filled wave costs half as much.  Shared memory is one FIFO ring of 12
-// chunks; stage j uses barrier slot j & 3 with parity (j >> 2) & 1, and the
-// producer fills stage j once stage j - depth has been released (depth 4 for big,
-// 3 for small stages), which also holds across the change of kind.
+// number of pairs); the remaining slots are cut into small tiles and, last,
+// quarter tiles, in the combination of whole rounds that ends soonest (the host
+// decides).  Shared memory is one FIFO ring of 12 chunks; stage j uses barrier
+// slot j & 3 with parity (j >> 2) & 1, and the producer fills stage j once stage
+// j - depth has been released (depth 4 for big, 3 for small and quarter stages),
+// which also holds across the changes of kind.
 constexpr int kChunkBytes = BM * BK * 2;      // 16 KB: one 128-row, 64-column BF16 box
 constexpr int kChunks = 12;
 constexpr size_t kMixedSmemBytes =
     1024 + size_t(kChunks) * kChunkBytes + sizeof(Control) + 16 + size_t(kEpilogueWarps) * kStageWarpBytes;
 
 struct MixedTile {
-  int big;        // 1 = 512x256, 0 = 256x256
-  int blk, nt;    // virtual block (p.group blocks), n-tile
+  int big;        // 1 = 512x256, 0 = 256x256 or 256x128
+  int quarter;    // 1 = 256x128 (one 128-column half of a 256-column tile)
+  int blk, nt;    // virtual block (p.group blocks), n-tile (256 columns)
+  int col0;       // first output column of the tile
   int row0;       // first row of the pair's tile inside the virtual block
   int valid;
 };
 __device__ __forceinline__ MixedTile decode_mixed(const GemmParams& p, int t) {
   MixedTile m;
   int tb;
-  int half = 0;
+  int half = 0, nq = 0;
+  m.quarter = 0;
   if (t < p.n_big) {
     m.big = 1;
     tb = t;
   } else if (p.h_last == 2) {
     m.big = 0;
-    const int u = t - p.n_big;
-    tb = p.n_big + (u >> 1);
-    half = u & 1;
+    if (t < p.n_small_end) {
+      const int u = t - p.n_big;
+      tb = p.n_big + (u >> 1);
+      half = u & 1;
+    } else {
+      // the last slots of the launch as four 256x128 tiles each: the remainder then fills the pairs more evenly
+      const int u = t - p.n_small_end;
+      tb = p.n_big + ((p.n_small_end - p.n_big) >> 1) + (u >> 2);
+      half = (u >> 1) & 1;
+      nq = u & 1;
+      m.quarter = 1;
+    }
   } else {
     // A block's last 512-row slot holds at most 256 rows (then the launch has no 512x256 tiles): its second
     // half does not exist and is not numbered, so that every tile index is a tile and consecutive indices
@@ -707,6 +725,7 @@ __device__ __forceinline__ MixedTile decode_mixed(const GemmParams& p, int t) {
       m.nt = w - full;
     }
     m.row0 = mtb * (4 * BM) + half * (2 * BM);
+    m.col0 = m.nt * BN;
     m.valid = m.row0 < p.vrows;
     return m;
   }
@@ -716,7 +735,8 @@ __device__ __forceinline__ MixedTile decode_mixed(const GemmParams& p, int t) {
   const int mtb = w / p.tiles_n;
   m.nt = w - mtb * p.tiles_n;
   m.row0 = mtb * (4 * BM) + half * (2 * BM);
-  m.valid = m.row0 < p.vrows;
+  m.col0 = m.nt * BN + nq * (BN / 2);
+  m.valid = m.row0 < p.vrows && m.col0 < p.N;      // the second half of a ragged last column tile may not exist
   return m;
 }
 
@@ -751,7 +771,7 @@ struct MixedIter {
     blk1 = f1.blk;
     a_row = b0.a_row0 + f0.r0;
     a_row1 = b1.a_row0 + f1.r0;
-    b_row = tile.nt * BN + cta_rank * (BN / 2);
+    b_row = tile.col0 + cta_rank * (tile.quarter ? BN / 4 : BN / 2);  // this CTA's half of the tile's B rows
     am = (p.n_seg > 1) ? p.seg_rank[tile.blk][seg] : b0.a_map;      // segmented K: blocks are never grouped
     am1 = (p.n_seg > 1) ? am : b1.a_map;
     bm = (p.n_seg > 1) ? am : b0.b_map;                             // the blocks of a group share their B tensor
@@ -827,6 +847,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
           ready_t = it.t;
         }
         const int big = it.tile.big;
+        // A 512x256 stage (3 chunks) follows only stages of its own kind: four of them fill the ring.  A 256x256
+        // stage (4 chunks) or a 256x128 stage (3 chunks, possibly behind 4-chunk stages) overwrites nothing newer
+        // than the third stage before it.
         const uint32_t depth = big ? 4u : 3u;
         if (j >= depth) {
           const uint32_t r = j - depth;      // this stage's chunks are free once stage r has been released
@@ -834,7 +857,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
         }
         const uint32_t slot = j & 3u;
         const uint32_t full_addr = map_to_cta(smem_u32(&ctl->full[slot]), 0);
-        const int nchunks = big ? 3 : 4;
+        const int quarter = it.tile.quarter;
+        const int nchunks = (big || quarter) ? 3 : 4;
         if (leader) mbar_arrive_expect_tx(&ctl->full[slot], uint32_t(2 * nchunks * kChunkBytes));
         uint8_t* c0 = smem + ((chunk + 0) % kChunks) * kChunkBytes;
         uint8_t* c1 = smem + ((chunk + 1) % kChunks) * kChunkBytes;
@@ -854,6 +878,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
           tma_load_2d_pair_hint(c0, &p.a_maps[it.am], full_addr, kx, it.a_row, pol_a);
           tma_load_2d_pair_hint(c1, &p.a_maps[it.am1], full_addr, kx, it.a_row1, pol_a);
           load_b(c2, kx);
+        } else if (quarter) {
+          // 256x128 tile: two k-atoms of A (chunks 0, 1) and this CTA's 64 B rows of both atoms in the two halves
+          // of chunk 2 (8 KB boxes: 64 rows x 64 columns from the 64-row-box maps, or one 64x64 box of a [K][N] weight)
+          const int kx = it.kb * 2 * BK;
+          tma_load_2d_pair_hint(c0, &p.a_maps[it.am], full_addr, kx, it.a_row, pol_a);
+          tma_load_2d_pair_hint(c1, &p.a_maps[it.am], full_addr, kx + BK, it.a_row, pol_a);
+          if (p.b_mn_major) {
+            tma_load_2d_pair_hint(c2, &p.b_maps[it.bm], full_addr, it.b_row, kx, pol_b);
+            tma_load_2d_pair_hint(c2 + kBChunkMnBytes, &p.b_maps[it.bm], full_addr, it.b_row, kx + BK, pol_b);
+          } else {
+            tma_load_2d_pair_hint(c2, &p.b_maps_q[it.bm], full_addr, kx, it.b_row, pol_b);
+            tma_load_2d_pair_hint(c2 + kChunkBytes / 2, &p.b_maps_q[it.bm], full_addr, kx + BK, it.b_row, pol_b);
+          }
         } else {
           const int kx = it.kb * 2 * BK;
           uint8_t* c3 = smem + ((chunk + 3) % kChunks) * kChunkBytes;
@@ -877,6 +914,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
     // 32-lane loop costs a divergence per MMA and measurably slows the issue stream.
     if (leader && lane == 0) {
       const uint32_t idesc = umma_idesc_bf16_f32(2 * BM, BN) | (p.b_mn_major ? kUmmaIdescBMnMajor : 0u);
+      const uint32_t idesc_q = umma_idesc_bf16_f32(2 * BM, BN / 2) | (p.b_mn_major ? kUmmaIdescBMnMajor : 0u);
       const uint64_t desc0 = umma_smem_desc_sw128(smem_u32(smem));
       // B chunks: the same ring, but an N-contiguous chunk is two 8 KB sub-chunks and a k-step is 2048 bytes
       const uint64_t desc0b = p.b_mn_major ? umma_smem_desc_sw128_mn(smem_u32(smem), kBChunkMnBytes) : desc0;
@@ -982,6 +1020,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
           ++uses0;
           ++uses1;
         } else {
+          // 256x256: A atoms in chunks 0 and 1, B atoms in chunks 2 and 3.  256x128: the two B atoms (64 rows per CTA)
+          // share chunk 2, and the MMA is 128 columns wide.
+          const int quarter = tile.quarter;
+          const uint32_t idesc_t = quarter ? idesc_q : idesc;
           const uint32_t acc_a = tmem_base + buf * BN;
           int kb_in_seg = 0;
           for (int kb = 0; kb < n_kb; ++kb, ++j) {
@@ -994,21 +1036,22 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
             const uint64_t d0 = desc0 + uint64_t((((chunk + 0) % kChunks) * kChunkBytes) >> 4);
             const uint64_t d1 = desc0 + uint64_t((((chunk + 1) % kChunks) * kChunkBytes) >> 4);
             const uint64_t d2 = desc0b + uint64_t((((chunk + 2) % kChunks) * kChunkBytes) >> 4);
-            const uint64_t d3 = desc0b + uint64_t((((chunk + 3) % kChunks) * kChunkBytes) >> 4);
+            const uint64_t d3 = quarter ? d2 + uint64_t((kChunkBytes / 2) >> 4)
+                                        : desc0b + uint64_t((((chunk + 3) % kChunks) * kChunkBytes) >> 4);
             const uint32_t first = kb != 0 ? 1u : 0u;
             if (full_stage) {
 #pragma unroll
-              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc_a, d0 + uint64_t(k * 2), d2 + uint64_t(k * bk), idesc, k ? 1u : first);
+              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc_a, d0 + uint64_t(k * 2), d2 + uint64_t(k * bk), idesc_t, k ? 1u : first);
 #pragma unroll
-              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc_a, d1 + uint64_t(k * 2), d3 + uint64_t(k * bk), idesc, 1u);
+              for (int k = 0; k < BK / UMMA_K; ++k) umma_bf16_pair(acc_a, d1 + uint64_t(k * 2), d3 + uint64_t(k * bk), idesc_t, 1u);
             } else {
               for (int ks = 0; ks < tail; ++ks) {
                 const int k = ks & 3;
-                umma_bf16_pair(acc_a, ((ks >> 2) ? d1 : d0) + uint64_t(k * 2), ((ks >> 2) ? d3 : d2) + uint64_t(k * bk), idesc,
+                umma_bf16_pair(acc_a, ((ks >> 2) ? d1 : d0) + uint64_t(k * 2), ((ks >> 2) ? d3 : d2) + uint64_t(k * bk), idesc_t,
                                ks ? 1u : first);
               }
             }
-            chunk = (chunk + 4) % kChunks;
+            chunk = (chunk + (quarter ? 3 : 4)) % kChunks;
             umma_commit_pair(&ctl->empty[j & 3u], 0x3);
             if (++kb_in_seg == kb_seg) kb_in_seg = 0;
           }
@@ -1034,7 +1077,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
     for (int t = unit; ok && t < p.total_tiles; t += n_units) {
       const MixedTile tile = decode_mixed(p, t);
       if (!tile.valid) continue;
-      const int ncols = min(BN, p.N - tile.nt * BN);
+      const int ncols = min(tile.quarter ? BN / 2 : BN, p.N - tile.col0);
       const int n_acc = tile.big ? 2 : 1;
       for (int a = 0; a < n_acc && ok; ++a) {
         const uint32_t buf = tile.big ? uint32_t(a) : (small_rr & 1u);
@@ -1052,13 +1095,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_mixed_kernel(const __grid_co
         const int act = kAct ? p.activation : int(ACT_NONE);
         const int oshift = act == ACT_SWIGLU ? 1 : 0;
         const int ocols = ncols >> oshift;
-        __nv_bfloat16* orow = p.out[b.out_idx] + int64_t(b.out_row0 + row_in_block) * p.ldo + ((int64_t(tile.nt) * BN) >> oshift);
+        __nv_bfloat16* orow = p.out[b.out_idx] + int64_t(b.out_row0 + row_in_block) * p.ldo + (int64_t(tile.col0) >> oshift);
         const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
         const int first_row = row_in_block - lane;          // row of lane 0
         __nv_bfloat16* obase = orow - int64_t(lane) * p.ldo;
         // 1) The whole accumulator row (256 columns) goes TMEM -> registers as packed BF16, then the
         //    accumulator is handed back at once: with two live accumulators per tile the MMA issuer
         //    waits for this, so the time TMEM is held matters more than the time the stores take.
+        //    (A 256x128 tile uses the first 128 columns; the rest is read too and never stored.)
         uint32_t packed[BN / 2];
 #pragma unroll
         for (int c = 0; c < BN / 64; ++c) {
@@ -1400,8 +1444,35 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
     p.n_big = use_big ? (total_big / info->max_pairs) * info->max_pairs : 0;
     p.h_last = (rows - (p.big_tiles_m - 1) * 4 * BM > 2 * BM) ? 2 : 1;
     p.vrows = rows;
-    p.total_tiles = p.h_last == 2 ? p.n_big + 2 * (total_big - p.n_big)
-                                  : n_vblocks * (2 * (p.big_tiles_m - 1) + 1) * p.tiles_n;
+    if (p.h_last == 2) {
+      // The slots left after the whole waves of 512x256 tiles are cut into 256x256 tiles (two per slot, half a big
+      // tile's time each) and, last, 256x128 tiles (four per slot; their stages carry 48 KB of operands for half the
+      // MMA work, so they are bound by operand delivery: measured 0.42 of a big tile's time each), in the combination
+      // of whole rounds over the pairs that ends soonest.
+      const int remaining = total_big - p.n_big;
+      int small_slots = remaining;
+      if (p.n_big > 0 && remaining > 0) {
+        const int pairs = info->max_pairs;
+        double best = 1e30;
+        for (int r1 = (2 * remaining + pairs - 1) / pairs; r1 >= 0; --r1) {
+          const int s_slots = std::min(remaining, (r1 * pairs) / 2);
+          const int r2 = (4 * (remaining - s_slots) + pairs - 1) / pairs;
+          const double cost = 0.5 * r1 + 0.42 * r2;
+          if (cost < best - 1e-9) {
+            best = cost;
+            small_slots = s_slots;
+          }
+        }
+      }
+      p.n_small_end = p.n_big + 2 * small_slots;
+      p.total_tiles = p.n_small_end + 4 * (remaining - small_slots);
+      if (remaining > small_slots && !L.b_mn_major)
+        for (int i = 0; i < L.n_b; ++i)
+          if (!encode_kmajor(&p.b_maps_q[i], L.b_ptr[i], L.N, L.K, BN / 4)) return record_cuda_error(cudaErrorUnknown);
+    } else {
+      p.total_tiles = n_vblocks * (2 * (p.big_tiles_m - 1) + 1) * p.tiles_n;
+      p.n_small_end = p.total_tiles;
+    }
     p.kb_big = int32_t((L.K + BK - 1) / BK);
     p.tail_big = int32_t((L.K - int64_t(p.kb_big - 1) * BK + UMMA_K - 1) / UMMA_K);
   }

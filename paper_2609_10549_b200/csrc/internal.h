@@ -77,6 +77,7 @@ constexpr int kMaxAMaps = 2 * kMaxP;   // shards plus, for the push variant, the
 struct GemmParams {
   CUtensorMap a_maps[kMaxAMaps];
   CUtensorMap b_maps[kMaxP];
+  CUtensorMap b_maps_q[kMaxP];   // the same B tensors with boxes of 64 rows (256x128 tiles: 64 B rows per CTA)
   __nv_bfloat16* out[kMaxP];
   int64_t ldo;             // output row pitch in elements
   int32_t n_blocks;
@@ -95,8 +96,10 @@ struct GemmParams {
   int32_t frags_m;         // 128-row fragments per block: ceil(rows_per_block / 128)
   int32_t tiles_m, tiles_n; // tiles per virtual block
   int32_t total_tiles;
-  // mixed-tile pair kernel: tiles [0, n_big) are 512x256, the rest 256x256 (two per remaining big tile)
+  // mixed-tile pair kernel: tiles [0, n_big) are 512x256, tiles [n_big, n_small_end) 256x256 (two per remaining
+  // 512x256 slot), tiles [n_small_end, total_tiles) 256x128 (four per slot)
   int32_t n_big;
+  int32_t n_small_end;
   int32_t big_tiles_m;     // 512-row tiles per block
   int32_t h_last;          // 256-row halves of a block's last 512-row slot that hold rows: 2, or 1 when at most 256 rows are left
   int32_t kb_big;          // 64-wide k-stages per segment of a big tile

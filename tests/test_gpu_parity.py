@@ -300,10 +300,31 @@ def test_small_slices_interdecom(op, P, m, N, K, d):
     (wl.OP_GEMM_RS, 4, 1024, 2568, 104, api.ORDER_RANK_MAJOR),     # 4 segments x 2 stages, every segment with a partial stage
 ])
 def test_big_and_small_tiles_in_one_launch(op, P, m, N, K, order):
+    _tile_mix_case(op, P, m, N, K, order)
+
+
+# Launches whose remainder after the whole waves of 512x256 tiles is planned with 256x128 tiles as well (on the 74 CTA
+# pairs of a B200: 14 of 384 slots left -> 56 tiles of 256x128; 46 of 416 left, last column tile ragged -> 74 tiles of
+# 256x256 and 36 of 256x128, some of whose second halves do not exist; 38 of 112 left in a segmented-K launch), both
+# weight layouts; element by element.
+@pytest.mark.parametrize("op,P,m,N,K,order,layout", [
+    (wl.OP_AG_GEMM, 4, 1024, 3072, 200, api.ORDER_RANK_MAJOR, api.B_NK),
+    (wl.OP_AG_GEMM, 4, 1024, 3080, 328, api.ORDER_STEP_MAJOR, api.B_NK),
+    (wl.OP_GEMM_RS, 8, 1024, 1544, 88, api.ORDER_RANK_MAJOR, api.B_NK),
+    (wl.OP_AG_GEMM, 4, 1024, 3072, 72, api.ORDER_RANK_MAJOR, api.B_KN),
+    (wl.OP_AG_GEMM, 4, 1024, 3080, 136, api.ORDER_RANK_MAJOR, api.B_KN),
+    (wl.OP_GEMM_RS, 4, 1024, 4096, 64, api.ORDER_RANK_MAJOR, api.B_NK),       # 54 of 128 slots left: one round of each kind
+])
+def test_three_tile_sizes_in_one_launch(op, P, m, N, K, order, layout):
+    _tile_mix_case(op, P, m, N, K, order, layout)
+
+
+def _tile_mix_case(op, P, m, N, K, order, layout=api.B_NK):
     w = small(op, P, m, N, K, dist=0.05)
     A_bits, B_bits = wl.make_inputs(w)
-    pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, order=order)
-    A, B = gu.device_inputs(A_bits, B_bits)
+    pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, order=order, b_layout=layout)
+    A = [api.to_device(a) for a in A_bits]
+    B = [api.to_device(np.ascontiguousarray(b.T) if layout == api.B_KN else b) for b in B_bits]
     outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
     ws = api.alloc_workspace(pr)
     (api.compass_ag_gemm if op == wl.OP_AG_GEMM else api.compass_gemm_rs)(pr, A, B, [o.view for o in outs], ws)
