@@ -39,8 +39,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + written) per launch of the GEMM kernel: dram__bytes_read.sum + dram__bytes_write.sum of one
 # ncu capture of `bench.py --steps 1 --warmup 3 --no-cpu-baseline --no-sweep`; the summary that holds the figures is
 # named beside them.  They are constants of that capture, not something this run measures.
-NCU_TRAFFIC = {"C2": {"bytes": 362.6e6, "source": "profiles/gemm_mixed_kernel_C2_C3.md"},
-               "C3": {"bytes": 799.0e6, "source": "profiles/gemm_mixed_kernel_C2_C3.md"}}
+NCU_TRAFFIC = {"C2": {"bytes": 360.6e6, "source": "profiles/gemm_mixed_kernel_C2_C3.md"},
+               "C3": {"bytes": 819.6e6, "source": "profiles/gemm_mixed_kernel_C2_C3.md"}}
 CALIBRATION_FILE = os.path.join(ROOT, "paper_2609_10549_b200", "calibration", "calib_b200.json")
 
 
