@@ -369,6 +369,25 @@ int compass_read_status(void* workspace, void* cuda_stream, int* detail);
  * the clock it was obtained at.  A measurement aid, not part of the paper's
  * method; both values are 0 before the first launch. */
 int compass_read_kernel_clock(void* workspace, void* cuda_stream, uint64_t* sm_cycles, uint64_t* nanoseconds);
+/* How a launch is cut into tiles (a diagnostic view of host-side planning; no
+ * GPU is touched).  decomposed = 0: the fused launch of problem->op (and
+ * rs_variant, order, rings); decomposed != 0: one sub-GEMM of compass_decomp
+ * with problem->d.  cta_pairs: how many clusters of two CTAs are resident at
+ * once (74 on a B200; 0 = no clusters: single-CTA tiles).  Blocks of at least
+ * 256 rows -- or groups of smaller blocks that share a weight tensor -- are
+ * computed by CTA pairs: 512x256 tiles for the whole waves of pairs, then
+ * 256x256 and 256x128 tiles for what is left, in whole rounds; the ring
+ * read-modify-write variant uses 256x256 tiles only; what cannot be paired
+ * runs as 128x256 tiles on single CTAs. */
+typedef struct compass_tile_counts {
+  int32_t cta_pairs;         /* 1: tiles computed by pairs of CTAs, 0: by single CTAs */
+  int32_t blocks;            /* blocks (contiguous output row ranges) of the launch */
+  int32_t rows_per_block;
+  int32_t blocks_per_group;  /* consecutive blocks tiled together (1 = none) */
+  int32_t tiles_512x256, tiles_256x256, tiles_256x128, tiles_128x256;
+  int32_t total_tiles;
+} compass_tile_counts;
+int compass_tile_plan(const compass_problem* problem, int decomposed, int cta_pairs, compass_tile_counts* out);
 /* The blocks of the fused launch for this problem, in launch order. */
 int compass_launch_plan(const compass_problem* problem, compass_plan_block* out, size_t capacity, size_t* count);
 /* End-to-end convenience with HOST tensors: copies A and B (host pointers,

@@ -38,7 +38,7 @@ EXPORTS = (
     "compass_read_status", "compass_launch_plan", "compass_fused_host", "compass_status_string",
     "compass_last_cuda_error", "compass_kernel_launch_count", "compass_gemm_rs_sequential_noalloc",
     "compass_set_wait_limit_us", "compass_calib_fit_line", "compass_ag_gemm_push", "compass_read_kernel_clock",
-    "compass_mlp_workspace_bytes", "compass_mlp_block", "compass_noalloc_read_status", "compass_select_ex", "compass_test_drop_flag_writes", "compass_tensor_map_cache_stats", "compass_decomp_comm",
+    "compass_mlp_workspace_bytes", "compass_mlp_block", "compass_noalloc_read_status", "compass_select_ex", "compass_test_drop_flag_writes", "compass_tensor_map_cache_stats", "compass_decomp_comm", "compass_tile_plan",
 )
 
 
@@ -72,6 +72,11 @@ class Calib(C.Structure):
 class Choice(C.Structure):
     _fields_ = [("strategy", C.c_int32), ("d_star", C.c_int32), ("t_fusion", C.c_double), ("t_decomp", C.c_double),
                 ("t_comp", C.c_double), ("t_comm", C.c_double), ("lam", C.c_double), ("t_star", C.c_double)]
+
+
+class TileCounts(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("cta_pairs", "blocks", "rows_per_block", "blocks_per_group", "tiles_512x256",
+                                          "tiles_256x256", "tiles_256x128", "tiles_128x256", "total_tiles")]
 
 
 class PlanBlock(C.Structure):
@@ -115,6 +120,7 @@ def lib() -> C.CDLL:
         L.compass_read_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]
         L.compass_read_kernel_clock.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
         L.compass_launch_plan.argtypes = [C.POINTER(Problem), C.POINTER(PlanBlock), C.c_size_t, C.POINTER(C.c_size_t)]
+        L.compass_tile_plan.argtypes = [C.POINTER(Problem), C.c_int, C.c_int, C.POINTER(TileCounts)]
         L.compass_fused_host.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t),
                                          C.c_void_p, C.c_size_t, C.c_void_p]
         L.compass_gemm_rs_sequential_noalloc.argtypes = [C.POINTER(Problem), pp, pp, pp, C.c_void_p]
@@ -244,6 +250,12 @@ def compass_workspace_bytes(problem: Problem, which: int = WS_FUSED) -> int:
     n = C.c_size_t(0)
     _check(lib().compass_workspace_bytes(C.byref(problem), which, C.byref(n)), "compass_workspace_bytes")
     return int(n.value)
+
+
+def compass_tile_plan(problem: Problem, decomposed: bool = False, cta_pairs: int = 74) -> TileCounts:
+    out = TileCounts()
+    _check(lib().compass_tile_plan(C.byref(problem), int(decomposed), int(cta_pairs), C.byref(out)), "compass_tile_plan")
+    return out
 
 
 def compass_launch_plan(problem: Problem) -> List[PlanBlock]:

@@ -526,6 +526,38 @@ extern "C" int compass_launch_plan(const compass_problem* pr, compass_plan_block
   return COMPASS_OK;
 }
 
+extern "C" int compass_tile_plan(const compass_problem* pr, int decomposed, int cta_pairs, compass_tile_counts* out) {
+  if (out == nullptr || cta_pairs < 0) return COMPASS_ERR_INVALID_ARG;
+  int st = validate_problem(pr, -1, decomposed != 0);
+  if (st != COMPASS_OK) return st;
+  static thread_local GemmLaunch L;
+  if (decomposed) {
+    // one sub-GEMM of compass_decomp: P x P blocks of (M/P)/d rows, a rank's P blocks adjacent
+    if (pr->d > 16) return COMPASS_ERR_UNSUPPORTED;
+    L = GemmLaunch{};
+    L.n_blocks = pr->P * pr->P;
+    L.rows_per_block = int(pr->M / pr->P / pr->d);
+    L.share_run = pr->P;
+    L.N = pr->N;
+    L.K = pr->K;
+  } else {
+    L.mode = GEMM_MODE_AUTO;
+    st = plan_fused(pr, &L, nullptr);
+    if (st != COMPASS_OK) return st;
+  }
+  const TilePlan t = plan_tiles(L, cta_pairs);
+  out->cta_pairs = t.pair;
+  out->blocks = L.n_blocks;
+  out->rows_per_block = L.rows_per_block;
+  out->blocks_per_group = t.group;
+  out->tiles_512x256 = t.mixed ? t.n_big : 0;
+  out->tiles_256x256 = t.pair ? (t.mixed ? t.n_small : t.total_tiles) : 0;
+  out->tiles_256x128 = t.mixed ? t.n_quarter : 0;
+  out->tiles_128x256 = t.pair ? 0 : t.total_tiles;
+  out->total_tiles = t.total_tiles;
+  return COMPASS_OK;
+}
+
 extern "C" int compass_ag_gemm(const compass_problem* pr, const void* const* A, const void* const* B, void* const* C,
                                void* ws, size_t ws_bytes, void* stream) {
   return fused_call(pr, COMPASS_OP_AG_GEMM, A, B, C, ws, ws_bytes, stream);

@@ -1337,40 +1337,75 @@ int gemm_tile_rows(int mode, int rows_per_block) {
   return pair ? 2 * BM : BM;
 }
 
-namespace {
-
-// How the blocks of a launch are tiled: `group` consecutive blocks (padded to sub_pad rows each) per virtual
-// block, and whether the virtual blocks are cut into 256-row tiles for CTA pairs or 128-row tiles for single CTAs.
-struct Tiling {
-  int group, sub_pad;
-  bool pair;
-};
-Tiling choose_tiling(const GemmLaunch& L) {
-  Tiling t;
+// How the blocks of a launch are tiled (pure host arithmetic; see TilePlan in internal.h).
+TilePlan plan_tiles(const GemmLaunch& L, int max_pairs) {
+  TilePlan t = {};
   t.sub_pad = (L.rows_per_block + BM - 1) / BM * BM;
   t.group = 1;
-  if (L.mode == GEMM_MODE_SINGLE) {
-    t.pair = false;
+  if (L.mode == GEMM_MODE_SINGLE || max_pairs <= 0) {
+    t.pair = 0;
   } else if (L.mode == GEMM_MODE_PAIR || t.sub_pad >= 2 * BM) {
-    t.pair = true;
+    t.pair = 1;
   } else {
     // One 128-row fragment per block: a CTA pair takes fragments of `group` consecutive blocks that read the
     // same B tensor (for the fused operators: the two ring entries of one step of a rank, adjacent in that
     // rank's schedule order).  Segmented K cannot group: its blocks walk the B tensors in different orders.
-    t.pair = false;
+    t.pair = 0;
     if (L.n_seg == 1 && L.share_run >= 2 && L.n_blocks % L.share_run == 0) {
       for (int g = 2; g <= L.share_run; ++g)
         if (L.share_run % g == 0) {
           t.group = g;
-          t.pair = true;
+          t.pair = 1;
           break;
         }
     }
   }
+  const int tile_rows = t.pair ? 2 * BM : BM;
+  t.vrows = t.group * t.sub_pad;
+  t.n_vblocks = L.n_blocks / t.group;
+  t.tiles_m = (t.vrows + tile_rows - 1) / tile_rows;
+  t.tiles_n = int((L.N + BN - 1) / BN);
+  t.total_tiles = t.n_vblocks * t.tiles_m * t.tiles_n;
+  t.n_small = t.total_tiles;
+  // Mixed tiles: 512x256 for as many whole waves of pairs as the launch holds, smaller ones for the rest.
+  t.mixed = t.pair && L.epilogue == EPI_STORE && L.mode != GEMM_MODE_PAIR;
+  if (!t.mixed || t.total_tiles <= 0) return t;
+  // rows of a (virtual) block that hold data when it is cut into 256-row halves of 512-row slots
+  const int rows = t.group > 1 ? t.vrows : L.rows_per_block;
+  t.vrows = rows;
+  t.big_tiles_m = (rows + 4 * BM - 1) / (4 * BM);
+  const int total_big = t.n_vblocks * t.big_tiles_m * t.tiles_n;
+  const bool use_big = rows % (4 * BM) == 0;
+  t.n_big = use_big ? (total_big / max_pairs) * max_pairs : 0;
+  t.h_last = (rows - (t.big_tiles_m - 1) * 4 * BM > 2 * BM) ? 2 : 1;
+  if (t.h_last == 2) {
+    // The slots left after the whole waves of 512x256 tiles are cut into 256x256 tiles (two per slot, half a big
+    // tile's time each) and, last, 256x128 tiles (four per slot; their stages carry 48 KB of operands for half the
+    // MMA work, so they are bound by operand delivery: measured 0.42 of a big tile's time each), in the combination
+    // of whole rounds over the pairs that ends soonest.
+    const int remaining = total_big - t.n_big;
+    int small_slots = remaining;
+    if (t.n_big > 0 && remaining > 0) {
+      double best = 1e30;
+      for (int r1 = (2 * remaining + max_pairs - 1) / max_pairs; r1 >= 0; --r1) {
+        const int s_slots = std::min(remaining, (r1 * max_pairs) / 2);
+        const int r2 = (4 * (remaining - s_slots) + max_pairs - 1) / max_pairs;
+        const double cost = 0.5 * r1 + 0.42 * r2;
+        if (cost < best - 1e-9) {
+          best = cost;
+          small_slots = s_slots;
+        }
+      }
+    }
+    t.n_small = 2 * small_slots;
+    t.n_quarter = 4 * (remaining - small_slots);
+  } else {
+    // a block's last 512-row slot holds at most 256 rows: only the 256-row halves that exist are numbered
+    t.n_small = t.n_vblocks * (2 * (t.big_tiles_m - 1) + 1) * t.tiles_n;
+  }
+  t.total_tiles = t.n_big + t.n_small + t.n_quarter;
   return t;
 }
-
-}  // namespace
 
 int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   static thread_local GemmParams p;
@@ -1380,13 +1415,8 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   DeviceInfo* info = nullptr;
   int st = device_info(&info);
   if (st != COMPASS_OK) return st;
-  Tiling tiling = choose_tiling(L);
-  if (tiling.pair && info->max_pairs <= 0) {   // no room for clusters on this device: single-CTA tiles, no grouping needed
-    tiling.pair = false;
-    tiling.group = 1;
-  }
-  const bool pair = tiling.pair;
-  const int tile_rows = pair ? 2 * BM : BM;
+  const TilePlan tiling = plan_tiles(L, info->max_pairs);
+  const bool pair = tiling.pair != 0;
   const int b_box_rows = pair ? BN / 2 : BN;
   for (int i = 0; i < L.n_a; ++i)
     if (!encode_kmajor(&p.a_maps[i], L.a_ptr[i], L.a_map_rows[i] ? L.a_map_rows[i] : L.a_rows, L.K, BM))
@@ -1407,12 +1437,11 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   p.tail_ksteps = int32_t((k_tail + UMMA_K - 1) / UMMA_K);
   p.group = tiling.group;
   p.sub_pad = tiling.sub_pad;
-  p.vrows = tiling.group * tiling.sub_pad;
+  p.vrows = tiling.vrows;
   p.frags_m = tiling.sub_pad / BM;
-  const int n_vblocks = L.n_blocks / tiling.group;
-  p.tiles_m = (p.vrows + tile_rows - 1) / tile_rows;
-  p.tiles_n = int32_t((L.N + BN - 1) / BN);
-  p.total_tiles = n_vblocks * p.tiles_m * p.tiles_n;
+  p.tiles_m = tiling.tiles_m;
+  p.tiles_n = tiling.tiles_n;
+  p.total_tiles = tiling.total_tiles;
   p.epilogue = L.epilogue;
   p.last_step = L.last_step;
   p.wait_limit_us = L.wait_limit_us ? L.wait_limit_us : (default_wait_limit_us() ? default_wait_limit_us() : 2000000u);
@@ -1433,48 +1462,17 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
       for (int s = 0; s < L.n_seg; ++s) p.seg_rank[b][s] = L.seg_rank[b][s];
 
   if (p.total_tiles <= 0) return COMPASS_OK;
-  // Mixed tiles: 512x256 for as many whole waves of pairs as the launch holds, 256x256 for the rest.
-  const bool mixed = pair && L.epilogue == EPI_STORE && L.mode != GEMM_MODE_PAIR;
+  const bool mixed = tiling.mixed != 0;
   if (mixed) {
-    // rows of a (virtual) block that hold data when it is cut into 256-row halves of 512-row slots
-    const int rows = tiling.group > 1 ? p.vrows : L.rows_per_block;
-    p.big_tiles_m = (rows + 4 * BM - 1) / (4 * BM);
-    const int total_big = n_vblocks * p.big_tiles_m * p.tiles_n;
-    const bool use_big = rows % (4 * BM) == 0;
-    p.n_big = use_big ? (total_big / info->max_pairs) * info->max_pairs : 0;
-    p.h_last = (rows - (p.big_tiles_m - 1) * 4 * BM > 2 * BM) ? 2 : 1;
-    p.vrows = rows;
-    if (p.h_last == 2) {
-      // The slots left after the whole waves of 512x256 tiles are cut into 256x256 tiles (two per slot, half a big
-      // tile's time each) and, last, 256x128 tiles (four per slot; their stages carry 48 KB of operands for half the
-      // MMA work, so they are bound by operand delivery: measured 0.42 of a big tile's time each), in the combination
-      // of whole rounds over the pairs that ends soonest.
-      const int remaining = total_big - p.n_big;
-      int small_slots = remaining;
-      if (p.n_big > 0 && remaining > 0) {
-        const int pairs = info->max_pairs;
-        double best = 1e30;
-        for (int r1 = (2 * remaining + pairs - 1) / pairs; r1 >= 0; --r1) {
-          const int s_slots = std::min(remaining, (r1 * pairs) / 2);
-          const int r2 = (4 * (remaining - s_slots) + pairs - 1) / pairs;
-          const double cost = 0.5 * r1 + 0.42 * r2;
-          if (cost < best - 1e-9) {
-            best = cost;
-            small_slots = s_slots;
-          }
-        }
-      }
-      p.n_small_end = p.n_big + 2 * small_slots;
-      p.total_tiles = p.n_small_end + 4 * (remaining - small_slots);
-      if (remaining > small_slots && !L.b_mn_major)
-        for (int i = 0; i < L.n_b; ++i)
-          if (!encode_kmajor(&p.b_maps_q[i], L.b_ptr[i], L.N, L.K, BN / 4)) return record_cuda_error(cudaErrorUnknown);
-    } else {
-      p.total_tiles = n_vblocks * (2 * (p.big_tiles_m - 1) + 1) * p.tiles_n;
-      p.n_small_end = p.total_tiles;
-    }
+    p.big_tiles_m = tiling.big_tiles_m;
+    p.n_big = tiling.n_big;
+    p.n_small_end = tiling.n_big + tiling.n_small;
+    p.h_last = tiling.h_last;
     p.kb_big = int32_t((L.K + BK - 1) / BK);
     p.tail_big = int32_t((L.K - int64_t(p.kb_big - 1) * BK + UMMA_K - 1) / UMMA_K);
+    if (tiling.n_quarter > 0 && !L.b_mn_major)
+      for (int i = 0; i < L.n_b; ++i)
+        if (!encode_kmajor(&p.b_maps_q[i], L.b_ptr[i], L.N, L.K, BN / 4)) return record_cuda_error(cudaErrorUnknown);
   }
   cudaError_t e;
   if (pair) {

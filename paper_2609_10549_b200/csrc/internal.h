@@ -153,7 +153,23 @@ struct GemmLaunch {
   uint32_t flag_token = 0;
 };
 
+// How a launch is cut into tiles, decided on the host from the block list and the number of co-resident CTA pairs.
+struct TilePlan {
+  int32_t pair;          // 1: clusters of two CTAs (256-row tiles); 0: single CTAs (128-row tiles)
+  int32_t mixed;         // 1: the mixed-tile kernel (512x256 / 256x256 / 256x128 tiles), plain-store epilogue
+  int32_t group;         // consecutive blocks tiled together (blocks below 256 rows that share a B tensor)
+  int32_t sub_pad;       // rows of a block rounded up to a multiple of 128
+  int32_t vrows;         // rows of a virtual block that are cut into tiles
+  int32_t n_vblocks;
+  int32_t tiles_m, tiles_n;
+  int32_t big_tiles_m;   // 512-row slots per virtual block (mixed only)
+  int32_t h_last;        // 256-row halves of a block's last slot that hold rows (mixed only)
+  int32_t n_big, n_small, n_quarter;   // tiles of 512x256, 256x256 (or 128x256 when pair == 0), 256x128
+  int32_t total_tiles;
+};
+
 // gemm_sm100.cu
+TilePlan plan_tiles(const GemmLaunch& launch, int max_pairs);
 int launch_gemm(const GemmLaunch& launch, cudaStream_t stream);
 size_t gemm_smem_bytes();
 void tensor_map_cache_stats(uint64_t* hits, uint64_t* misses);
