@@ -77,8 +77,10 @@ enum { COMPASS_DTYPE_BF16 = 0 };
  *     schedule order and added into the owner's rows in ring order by a
  *     vectorised read-modify-write in the GEMM epilogue.  The running sum lives
  *     in the BF16 output rows (what a BF16 ring transfer would carry), so the
- *     result is rounded once per contributor; the owner's contribution,
- *     scheduled last, completes it.  Needs one int32 counter per output tile in
+ *     result is rounded once per contributor (the per-element error grows
+ *     like sqrt(P): within 1e-2 * max|result| + 1e-3 for P <= 8, exceeded by
+ *     rare elements at P = 16); the owner's contribution, scheduled last,
+ *     completes it.  Needs one int32 counter per output tile in
  *     the workspace (zero before the first call; every call leaves them zero,
  *     unless it reported COMPASS_ERR_TIMEOUT: then re-initialise the workspace). */
 enum { COMPASS_RS_SEGMENTED_K = 0, COMPASS_RS_RING_RMW = 1 };
