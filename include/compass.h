@@ -83,7 +83,13 @@ enum { COMPASS_DTYPE_BF16 = 0 };
  *     completes it.  Needs one int32 counter per output tile in
  *     the workspace (zero before the first call; every call leaves them zero,
  *     unless it reported COMPASS_ERR_TIMEOUT: then re-initialise the workspace). */
-enum { COMPASS_RS_SEGMENTED_K = 0, COMPASS_RS_RING_RMW = 1 };
+/*   RING_RMW_F32: the same ordered ring accumulation with the running sum kept
+ *     in FP32 scratch inside the workspace (what an FP32 ring transfer would
+ *     carry: twice the bytes per hop): contributors add their FP32 partial
+ *     tile to it in ring order and the owner's contribution, last, writes the
+ *     BF16 result -- one rounding, whatever P.  Needs the tile counters of
+ *     RING_RMW plus P * (M/P) * N * 4 bytes in the workspace. */
+enum { COMPASS_RS_SEGMENTED_K = 0, COMPASS_RS_RING_RMW = 1, COMPASS_RS_RING_RMW_F32 = 2 };
 enum { COMPASS_STRATEGY_INTRAFUSION = 0, COMPASS_STRATEGY_INTERDECOM = 1 };
 /* Launch order of the fused kernels.  Every rank's tiles are always issued in
  * that rank's schedule order (step ascending, ring 0 before ring 1).  What the
@@ -93,7 +99,7 @@ enum { COMPASS_STRATEGY_INTRAFUSION = 0, COMPASS_STRATEGY_INTERDECOM = 1 };
  *     shard stays in L2 while it is used; default);
  *   STEP_MAJOR: all ranks advance in lockstep: step 0 of every rank, then
  *     step 1, ... (what P GPUs running concurrently would do).
- * The ring read-modify-write variant always uses STEP_MAJOR (its ordered adds
+ * The ring read-modify-write variants always use STEP_MAJOR (its ordered adds
  * need contributor s of a partition to precede contributor s+1 in the launch);
  * the segmented-K variant has one block per partition and ignores the field. */
 enum { COMPASS_ORDER_RANK_MAJOR = 0, COMPASS_ORDER_STEP_MAJOR = 1 };
@@ -227,7 +233,7 @@ int compass_ag_gemm_push(const compass_problem* problem, const void* const* A, c
  * would travel the ring, ending with the owner c.
  *   A: P device pointers [M x K];  B: P device pointers [N x K];
  *   Out: P device pointers [M/P x N] (every element is written).
- * Precondition of COMPASS_RS_RING_RMW: contributor s of an output tile waits,
+ * Precondition of COMPASS_RS_RING_RMW and COMPASS_RS_RING_RMW_F32: contributor s of an output tile waits,
  * holding its SM, for contributor s-1, which is earlier in the launch; that
  * is deadlock-free because all CTAs of the launch are resident at once, and
  * the grid is sized for an otherwise idle GPU.  Run nothing else on the GPU's

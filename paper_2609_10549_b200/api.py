@@ -20,7 +20,7 @@ ERR_SCRATCH_LIMIT = 8
 NOALLOC_SCRATCH_BYTES = 32 * 1024 * 1024
 OP_AG_GEMM, OP_GEMM_RS = 0, 1
 DTYPE_BF16 = 0
-RS_SEGMENTED_K, RS_RING_RMW = 0, 1
+RS_SEGMENTED_K, RS_RING_RMW, RS_RING_RMW_F32 = 0, 1, 2
 STRATEGY_INTRAFUSION, STRATEGY_INTERDECOM = 0, 1
 ORDER_RANK_MAJOR, ORDER_STEP_MAJOR = 0, 1
 COPY_KERNEL, COPY_ENGINES = 0, 1

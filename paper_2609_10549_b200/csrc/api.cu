@@ -28,7 +28,8 @@ int validate_problem(const compass_problem* pr, int want_op, bool need_d) {
   if (need_d && pr->d < 1) return COMPASS_ERR_INVALID_ARG;
   if (pr->order != COMPASS_ORDER_RANK_MAJOR && pr->order != COMPASS_ORDER_STEP_MAJOR) return COMPASS_ERR_INVALID_ARG;
   if (pr->copy_mode != COMPASS_COPY_KERNEL && pr->copy_mode != COMPASS_COPY_ENGINES) return COMPASS_ERR_INVALID_ARG;
-  if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant != COMPASS_RS_SEGMENTED_K && pr->rs_variant != COMPASS_RS_RING_RMW)
+  if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant != COMPASS_RS_SEGMENTED_K && pr->rs_variant != COMPASS_RS_RING_RMW &&
+      pr->rs_variant != COMPASS_RS_RING_RMW_F32)
     return COMPASS_ERR_INVALID_ARG;
   if ((pr->b_layout != COMPASS_B_NK && pr->b_layout != COMPASS_B_KN) || pr->reserved != 0) return COMPASS_ERR_INVALID_ARG;
   if (pr->dtype != COMPASS_DTYPE_BF16 || pr->P > COMPASS_MAX_P) return COMPASS_ERR_UNSUPPORTED;
@@ -176,7 +177,7 @@ void plan_rs_ring(const compass_problem* pr, const compass_sched_entry* table, G
   L->n_seg = 1;
   L->rows_per_block = int(m / rings);
   L->share_run = rings;  // a rank's two ring entries of one step are adjacent and multiply by the same B_rank
-  L->epilogue = EPI_RING_RMW;
+  L->epilogue = pr->rs_variant == COMPASS_RS_RING_RMW_F32 ? EPI_RING_RMW_F32 : EPI_RING_RMW;
   L->last_step = P - 1;
   int n = 0;
   for (int step = 0; step < P; ++step)
@@ -223,6 +224,15 @@ int plan_fused(const compass_problem* pr, GemmLaunch* L, compass_plan_block* vie
   return COMPASS_OK;
 }
 
+// FP32 running sums of the ring read-modify-write variant with FP32 scratch: behind the tile counters, one per owner.
+void set_running_sums(const compass_problem* pr, GemmLaunch* L, void* ws) {
+  for (int r = 0; r < kMaxP; ++r) L->sum_ptr[r] = nullptr;
+  if (pr->op != COMPASS_OP_GEMM_RS || pr->rs_variant != COMPASS_RS_RING_RMW_F32) return;
+  uint8_t* base = static_cast<uint8_t*>(ws) + COMPASS_STATUS_BYTES + align_up(rmw_counter_count(pr) * sizeof(int32_t));
+  const size_t per_owner = align_up(size_t(pr->M / pr->P) * size_t(pr->N) * sizeof(float));
+  for (int r = 0; r < pr->P; ++r) L->sum_ptr[r] = reinterpret_cast<float*>(base + size_t(r) * per_owner);
+}
+
 int fused_call(const compass_problem* pr, int op, const void* const* A, const void* const* B, void* const* out, void* ws,
                size_t ws_bytes, void* stream) {
   int st = validate_problem(pr, op, false);
@@ -241,6 +251,7 @@ int fused_call(const compass_problem* pr, int op, const void* const* A, const vo
   }
   L.status = static_cast<StatusBlock*>(ws);
   L.tile_counters = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + COMPASS_STATUS_BYTES);
+  set_running_sums(pr, &L, ws);
   return launch_gemm(L, static_cast<cudaStream_t>(stream));
 }
 
@@ -466,8 +477,10 @@ extern "C" int compass_workspace_bytes(const compass_problem* pr, int which, siz
   if (st != COMPASS_OK) return st;
   size_t total = COMPASS_STATUS_BYTES;
   if (which == COMPASS_WS_FUSED) {
-    if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant == COMPASS_RS_RING_RMW)
+    if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant != COMPASS_RS_SEGMENTED_K)
       total += align_up(rmw_counter_count(pr) * sizeof(int32_t));
+    if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant == COMPASS_RS_RING_RMW_F32)
+      total += size_t(pr->P) * align_up(size_t(pr->M / pr->P) * size_t(pr->N) * sizeof(float));
   } else if (which == COMPASS_WS_DECOMP) {
     const size_t inner = pr->op == COMPASS_OP_AG_GEMM ? size_t(pr->K) : size_t(pr->N);
     total += size_t(pr->P) * align_up(size_t(pr->M) * inner * 2);
@@ -513,7 +526,7 @@ extern "C" int compass_launch_plan(const compass_problem* pr, compass_plan_block
   if (count == nullptr) return COMPASS_ERR_INVALID_ARG;
   int st = validate_problem(pr, -1, false);
   if (st != COMPASS_OK) return st;
-  const bool per_entry = pr->op == COMPASS_OP_AG_GEMM || pr->rs_variant == COMPASS_RS_RING_RMW;
+  const bool per_entry = pr->op == COMPASS_OP_AG_GEMM || pr->rs_variant != COMPASS_RS_SEGMENTED_K;
   const size_t n = size_t(pr->rings) * pr->P * (per_entry ? pr->P : 1);
   *count = n;
   if (out == nullptr) return COMPASS_OK;
@@ -639,6 +652,7 @@ extern "C" int compass_mlp_block(const compass_mlp* mp, const void* const* X, co
   }
   L.status = static_cast<StatusBlock*>(ws);
   L.tile_counters = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + COMPASS_STATUS_BYTES);
+  set_running_sums(&rs, &L, ws);
   return launch_gemm(L, static_cast<cudaStream_t>(stream));
 }
 

@@ -258,7 +258,9 @@ struct StageIter {
 };
 
 // kAct: the plain-store epilogue applies p.activation (its own instantiation, see gemm_mixed_kernel).
-template <bool kPair, bool kAct>
+// kF32Sum: the ring read-modify-write epilogue keeps the running sum in FP32 scratch (p.sum) and only the last
+// contributor writes the BF16 output (again its own instantiation).
+template <bool kPair, bool kAct, bool kF32Sum>
 __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
   using C = Cfg<kPair>;
   extern __shared__ uint8_t smem_raw[];
@@ -494,6 +496,122 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       __nv_bfloat16* obase = p.out[b.out_idx] + int64_t(b.out_row0 + first_row) * p.ldo + ((int64_t(tc.nt) * BN) >> oshift);
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + buf * BN;
       const int npass = (ocols + 63) >> 6;
+
+      if constexpr (kF32Sum) {
+        // Ring read-modify-write with the running sum in FP32 scratch.  Same counters and ordering as below; the
+        // sum travels as 32-column pieces (128 bytes per row: 4 rows per load or store instruction, transposed
+        // through shared memory into one row per lane), four pieces in flight ahead of the one being added.
+        const bool live = frag.r0 < p.rows_per_block;          // a fragment past the block adds nothing
+        const bool add_previous = live && b.step > 0;
+        const bool last = int(b.step) == p.last_step;          // the owner's contribution: writes the BF16 result
+        int* counter = p.tile_counters + (int64_t(b.part) * p.frags_m + frag.r0 / BM) * p.tiles_n + tc.nt;
+        float* sbase = p.sum[b.out_idx] + int64_t(b.out_row0 + first_row) * p.N + int64_t(tc.nt) * BN;
+        uint4 ahead[4][8];
+        auto fetch = [&](int piece, uint4 (&dst)[8]) {
+          const int col = piece * 32 + seg * 4;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int r = i * 4 + (lane >> 3);
+            dst[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (first_row + r < p.rows_per_block && col < ncols)
+              dst[i] = __ldcg(reinterpret_cast<const uint4*>(sbase + int64_t(r) * p.N + col));
+          }
+        };
+        if (add_previous) {
+          int ready = 1;
+          if (lane == 0) ready = wait_counter(counter, int(b.step) * kEpilogueWarps, ctl, p, t) ? 1 : 0;
+          ready = __shfl_sync(0xffffffffu, ready, 0);
+          __syncwarp();      // orders the other lanes' loads behind lane 0's acquire
+          if (!ready) break;
+#pragma unroll
+          for (int piece = 0; piece < 4; ++piece) fetch(piece, ahead[piece]);
+        }
+        if (!wait_bounded(&ctl->acc_full[buf], acc_phase, ctl, p, WAIT_ACC_FULL, t)) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int c = 0; c < BN / 32; ++c) {
+          float prev[32];
+          if (add_previous) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              *reinterpret_cast<uint4*>(stage + (i * 4 + (lane >> 3)) * kStageRowBytes + seg * 16) = ahead[c & 3][i];
+            __syncwarp();
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+              const uint4 q = *reinterpret_cast<const uint4*>(stage + lane * kStageRowBytes + g * 16);
+              prev[g * 4 + 0] = __uint_as_float(q.x);
+              prev[g * 4 + 1] = __uint_as_float(q.y);
+              prev[g * 4 + 2] = __uint_as_float(q.z);
+              prev[g * 4 + 3] = __uint_as_float(q.w);
+            }
+            __syncwarp();
+            if (c + 4 < BN / 32) fetch(c + 4, ahead[c & 3]);
+          }
+          uint32_t v[32];
+          tmem_ld_32x32b_x32(taddr + c * 32, v);
+          tmem_ld_wait();
+          if (c == BN / 32 - 1) {
+            // accumulator fully copied to registers: hand it back to the MMA issuer
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+              if (kPair) mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->acc_empty[buf]), 0));
+              else mbar_arrive(&ctl->acc_empty[buf]);
+            }
+          }
+          if (add_previous) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + prev[i]);
+          }
+          if (c * 32 < ncols && live) {
+            if (last) {
+              // BF16 result: 64 bytes per row; every store instruction writes 8 rows x 64 contiguous bytes
+              uint4* srow = reinterpret_cast<uint4*>(stage + lane * kStageRowBytes);
+#pragma unroll
+              for (int g = 0; g < 4; ++g)
+                srow[g] = make_uint4(pack_bf16x2(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1])),
+                                     pack_bf16x2(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3])),
+                                     pack_bf16x2(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5])),
+                                     pack_bf16x2(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7])));
+              __syncwarp();
+              const int col = c * 32 + (lane & 3) * 8;
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int r = i * 8 + (lane >> 2);
+                if (first_row + r < p.rows_per_block && col < ncols)
+                  *reinterpret_cast<uint4*>(obase + int64_t(r) * p.ldo + col) =
+                      *reinterpret_cast<const uint4*>(stage + r * kStageRowBytes + (lane & 3) * 16);
+              }
+              __syncwarp();
+            } else {
+              // FP32 running sum: 128 bytes per row; every store instruction writes 4 rows x 128 contiguous bytes
+              uint4* srow = reinterpret_cast<uint4*>(stage + lane * kStageRowBytes);
+#pragma unroll
+              for (int g = 0; g < 8; ++g) srow[g] = make_uint4(v[g * 4 + 0], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
+              __syncwarp();
+              const int col = c * 32 + seg * 4;
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const int r = i * 4 + (lane >> 3);
+                if (first_row + r < p.rows_per_block && col < ncols)
+                  *reinterpret_cast<uint4*>(sbase + int64_t(r) * p.N + col) =
+                      *reinterpret_cast<const uint4*>(stage + r * kStageRowBytes + seg * 16);
+              }
+              __syncwarp();
+            }
+          }
+        }
+        if (live) {
+          // the warp barriers above ordered every lane's stores before lane 0's release of the counter
+          if (lane == 0) {
+            int before;
+            asm volatile("atom.add.release.gpu.global.s32 %0, [%1], 1;" : "=r"(before) : "l"(counter) : "memory");
+            // the last warp of the last contributor leaves the counter at zero for the next call
+            if (last && before == (p.last_step + 1) * kEpilogueWarps - 1) atomicExch(counter, 0);
+          }
+        }
+        continue;
+      }
 
       // Ring read-modify-write: contributor `step` of a partition adds its
       // partial tile to the running sum that contributor step-1 left in the
@@ -1287,13 +1405,17 @@ int device_info(DeviceInfo** out) {
   if (!info.ready) {
     e = cudaDeviceGetAttribute(&info.num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return record_cuda_error(e);
-    e = cudaFuncSetAttribute(gemm_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<false>()));
+    e = cudaFuncSetAttribute(gemm_kernel<false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<false>()));
     if (e != cudaSuccess) return record_cuda_error(e);
-    e = cudaFuncSetAttribute(gemm_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<false>()));
+    e = cudaFuncSetAttribute(gemm_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<false>()));
     if (e != cudaSuccess) return record_cuda_error(e);
-    e = cudaFuncSetAttribute(gemm_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<true>()));
+    e = cudaFuncSetAttribute(gemm_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<false>()));
     if (e != cudaSuccess) return record_cuda_error(e);
-    e = cudaFuncSetAttribute(gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<true>()));
+    e = cudaFuncSetAttribute(gemm_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<true>()));
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaFuncSetAttribute(gemm_kernel<true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<true>()));
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaFuncSetAttribute(gemm_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_bytes<true>()));
     if (e != cudaSuccess) return record_cuda_error(e);
     e = cudaFuncSetAttribute(gemm_mixed_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kMixedSmemBytes));
     if (e != cudaSuccess) return record_cuda_error(e);
@@ -1311,7 +1433,7 @@ int device_info(DeviceInfo** out) {
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int clusters = 0;
-    e = cudaOccupancyMaxActiveClusters(&clusters, gemm_kernel<true, false>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&clusters, gemm_kernel<true, false, false>, &cfg);
     if (e != cudaSuccess) return record_cuda_error(e);
     info.max_pairs = clusters;
     info.ready = true;
@@ -1411,6 +1533,7 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   static thread_local GemmParams p;
   // an activation goes with the plain store only (the ring read-modify-write adds partial sums)
   if (L.activation != ACT_NONE && L.epilogue != EPI_STORE) return COMPASS_ERR_INVALID_ARG;
+  if (L.epilogue == EPI_RING_RMW_F32 && L.n_out > 0 && L.sum_ptr[0] == nullptr) return COMPASS_ERR_INVALID_ARG;
   if (L.activation == ACT_SWIGLU && (L.N % 16 != 0 || L.ldo < L.N / 2)) return COMPASS_ERR_INVALID_ARG;
   DeviceInfo* info = nullptr;
   int st = device_info(&info);
@@ -1425,7 +1548,10 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
     if (L.b_mn_major ? !encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.K, L.N, 64)      // [K][N]: boxes of 64 columns x 64 k-rows
                      : !encode_kmajor(&p.b_maps[i], L.b_ptr[i], L.N, L.K, b_box_rows))
       return record_cuda_error(cudaErrorUnknown);
-  for (int i = 0; i < L.n_out; ++i) p.out[i] = static_cast<__nv_bfloat16*>(L.out_ptr[i]);
+  for (int i = 0; i < L.n_out; ++i) {
+    p.out[i] = static_cast<__nv_bfloat16*>(L.out_ptr[i]);
+    p.sum[i] = L.sum_ptr[i];
+  }
   p.ldo = L.ldo;
   p.n_blocks = L.n_blocks;
   p.rows_per_block = L.rows_per_block;
@@ -1491,12 +1617,14 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
     cfg.numAttrs = 1;
     if (mixed && L.activation != ACT_NONE) e = cudaLaunchKernelEx(&cfg, gemm_mixed_kernel<true>, p);
     else if (mixed) e = cudaLaunchKernelEx(&cfg, gemm_mixed_kernel<false>, p);
-    else if (L.activation != ACT_NONE) e = cudaLaunchKernelEx(&cfg, gemm_kernel<true, true>, p);
-    else e = cudaLaunchKernelEx(&cfg, gemm_kernel<true, false>, p);
+    else if (L.epilogue == EPI_RING_RMW_F32) e = cudaLaunchKernelEx(&cfg, gemm_kernel<true, false, true>, p);
+    else if (L.activation != ACT_NONE) e = cudaLaunchKernelEx(&cfg, gemm_kernel<true, true, false>, p);
+    else e = cudaLaunchKernelEx(&cfg, gemm_kernel<true, false, false>, p);
   } else {
     const int grid = p.total_tiles < info->num_sms ? p.total_tiles : info->num_sms;
-    if (L.activation != ACT_NONE) gemm_kernel<false, true><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);
-    else gemm_kernel<false, false><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);
+    if (L.epilogue == EPI_RING_RMW_F32) gemm_kernel<false, false, true><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);
+    else if (L.activation != ACT_NONE) gemm_kernel<false, true, false><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);
+    else gemm_kernel<false, false, false><<<grid, kThreads, smem_bytes<false>(), stream>>>(p);
     e = cudaGetLastError();
   }
   count_kernel_launch();

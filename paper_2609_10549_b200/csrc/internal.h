@@ -70,6 +70,7 @@ enum GemmMode : int32_t {
 enum EpilogueMode : int32_t {
   EPI_STORE = 0,      // round to BF16 and store
   EPI_RING_RMW = 1,   // ordered accumulate into the output in ring order
+  EPI_RING_RMW_F32 = 2,   // the same with the running sum in FP32 scratch; the last contributor writes the BF16 output
 };
 
 constexpr int kMaxAMaps = 2 * kMaxP;   // shards plus, for the push variant, the per-rank gather buffers
@@ -79,6 +80,7 @@ struct GemmParams {
   CUtensorMap b_maps[kMaxP];
   CUtensorMap b_maps_q[kMaxP];   // the same B tensors with boxes of 64 rows (256x128 tiles: 64 B rows per CTA)
   __nv_bfloat16* out[kMaxP];
+  float* sum[kMaxP];       // FP32 running sums, one [rows x N] tensor per output (EPI_RING_RMW_F32 only)
   int64_t ldo;             // output row pitch in elements
   int32_t n_blocks;
   int32_t rows_per_block;
@@ -126,6 +128,7 @@ struct GemmLaunch {
   int64_t a_map_rows[kMaxAMaps] = {};   // rows of A tensor i; 0 = a_rows
   const void* b_ptr[kMaxP];
   void* out_ptr[kMaxP];
+  float* sum_ptr[kMaxP] = {};   // FP32 running sums (EPI_RING_RMW_F32)
   int n_a = 0, n_b = 0, n_out = 0;
   int64_t a_rows = 0;      // rows of every A tensor
   int64_t K = 0;           // columns (contraction length) of every A and B tensor

@@ -5,8 +5,8 @@
     python -m paper_2609_10549_b200.run_case --op ag --variant decomp --d 4 --P 4 --M 4096 --N 3072 --K 4096
 
 --op ag|rs: AllGather+GEMM (N per rank, K full) or GEMM+ReduceScatter (K per rank, N full).
---variant fused|ring|push|decomp|comm: the fused kernel (gather by address / segmented K), the ring
-read-modify-write GEMM+ReduceScatter, the readiness-driven AllGather+GEMM, InterDecom with --d stages, or the --d
+--variant fused|ring|ring32|push|decomp|comm: the fused kernel (gather by address / segmented K), the ring
+read-modify-write GEMM+ReduceScatter (running sum in the BF16 output rows, or in FP32 scratch), the readiness-driven AllGather+GEMM, InterDecom with --d stages, or the --d
 sub-collectives of InterDecom alone (gather / reduce kernels on one stream; reported in GB/s of their algorithmic bytes).
 Inputs are drawn on the device (seeded); every launch is timed between its own pair of CUDA events on the
 launching stream after --warmup untimed launches.  Prints one JSON line: median / best milliseconds,
@@ -25,7 +25,7 @@ import numpy as np
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--op", choices=["ag", "rs"], required=True)
-    ap.add_argument("--variant", choices=["fused", "ring", "push", "decomp", "comm"], default="fused")
+    ap.add_argument("--variant", choices=["fused", "ring", "ring32", "push", "decomp", "comm"], default="fused")
     ap.add_argument("--P", type=int, required=True)
     ap.add_argument("--M", type=int, required=True)
     ap.add_argument("--N", type=int, required=True)
@@ -47,8 +47,8 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("run_case needs a CUDA device: the library has no CPU fallback")
     op = wl.OP_AG_GEMM if args.op == "ag" else wl.OP_GEMM_RS
-    if args.variant == "ring" and op != wl.OP_GEMM_RS:
-        raise SystemExit("--variant ring is a GEMM+ReduceScatter variant")
+    if args.variant in ("ring", "ring32") and op != wl.OP_GEMM_RS:
+        raise SystemExit("--variant ring / ring32 is a GEMM+ReduceScatter variant")
     if args.variant == "push" and op != wl.OP_AG_GEMM:
         raise SystemExit("--variant push is an AllGather+GEMM variant")
     w = wl.Workload("case", op, P=args.P, M=args.M, N=args.N, K=args.K)
@@ -60,12 +60,12 @@ def main():
     B = [mk(b_shape, args.b_std) for _ in range(w.P)]
     out = [torch.empty(w.out_shape, dtype=torch.bfloat16, device="cuda") for _ in range(w.P)]
     pr = api.make_problem(op, w.P, w.M, w.N, w.K, rings=args.rings, d=args.d,
-                          rs_variant=api.RS_RING_RMW if args.variant == "ring" else api.RS_SEGMENTED_K,
+                          rs_variant={"ring": api.RS_RING_RMW, "ring32": api.RS_RING_RMW_F32}.get(args.variant, api.RS_SEGMENTED_K),
                           order=api.ORDER_RANK_MAJOR if args.order == "rank" else api.ORDER_STEP_MAJOR,
                           b_layout=api.B_NK if args.layout == "nk" else api.B_KN)
     stream = torch.cuda.current_stream()
     side = torch.cuda.Stream()
-    if args.variant in ("fused", "ring"):
+    if args.variant in ("fused", "ring", "ring32"):
         ws = api.alloc_workspace(pr)
         call = api.compass_ag_gemm if op == wl.OP_AG_GEMM else api.compass_gemm_rs
         run = lambda: call(pr, A, B, out, ws, stream)

@@ -661,6 +661,45 @@ def test_config3_ring_rmw_every_element():
     check_every_element(w, outs, f"{w.name} ring-RMW", ring_rmw=True)
 
 
+# ---- ring read-modify-write with the running sum in FP32 scratch: one rounding, whatever P ------------------------------
+
+@pytest.mark.parametrize("P,m,N,K,rings", RS_SHAPES + [(16, 128, 264, 72, 2), (16, 64, 520, 200, 1), (8, 384, 776, 72, 2)])
+def test_gemm_rs_ring_f32_small_shapes(P, m, N, K, rings):
+    """Held to the single-rounding acceptance of the segmented-K variant (check_all: per-element rule and RMS <= 2^-8),
+    at P = 16 too, where the BF16 running sum of the plain ring variant gives out."""
+    w = small(wl.OP_GEMM_RS, P, m, N, K, dist=0.05)
+    A, B = wl.make_inputs(w)
+    outs, status, guards = gu.run_fused(w, A, B, rings=rings, rs_variant=api.RS_RING_RMW_F32)
+    assert status == (api.OK, 0) and guards
+    check_all(outs, ops.gemm_rs(A, B, rings=rings), w.name)
+
+
+def test_ring_f32_integers_exact_counters_return_to_zero_and_scratch_is_not_assumed_clean():
+    w = wl.Workload("ints-ring-f32", wl.OP_GEMM_RS, P=4, M=4 * 512, N=520, K=64)
+    A_bits, B_bits = wl.make_structured_inputs(w, "index")
+    pr = gu.problem_of(w, rs_variant=api.RS_RING_RMW_F32)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    ws = api.alloc_workspace(pr)
+    n_counters = 2 * w.P * (256 // 128) * 3                       # partitions x 128-row fragments x column tiles
+    ws[api.STATUS_BYTES + 4 * n_counters + 256:].fill_(0x7F)      # garbage (NaN patterns) in the FP32 scratch
+    ref = ops.gemm_rs(A_bits, B_bits)
+    for _ in range(2):
+        outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        api.compass_gemm_rs(pr, A, B, [o.view for o in outs], ws)
+        assert api.compass_read_status(ws) == (api.OK, 0)
+        for o, r in zip(outs, ref):
+            assert np.array_equal(ops.bf16_bits_to_f64(o.bits()), r)
+        assert int(ws[api.STATUS_BYTES:api.STATUS_BYTES + 4 * n_counters].view(torch.int32).abs().sum().item()) == 0
+
+
+def test_config3_ring_f32_every_element():
+    w = wl.C3_RS
+    A, B = _inputs(w)
+    outs, status, guards = gu.run_fused(w, A, B, rs_variant=api.RS_RING_RMW_F32)
+    assert status == (api.OK, 0) and guards
+    check_every_element(w, outs, f"{w.name} ring-RMW, FP32 running sum")      # single-rounding limits
+
+
 def test_bounded_wait_reports_timeout_and_the_context_survives():
     """A tile counter that no contributor will ever raise (the host plants a
     negative value) makes the ring epilogue's wait run out: the kernel must
@@ -903,6 +942,25 @@ def _random_cases(n, seed):
             continue
         cases.append((op, P, m, N, K, rings, int(rng.integers(0, 2)), int(rng.integers(0, 2)), int(rng.integers(0, 2))))
     return cases
+
+
+def _random_rs_cases(n, seed):
+    return [c for c in _random_cases(4 * n, seed) if c[0] == wl.OP_GEMM_RS][:n]
+
+
+@pytest.mark.parametrize("op,P,m,N,K,rings,order,variant,layout", _random_rs_cases(12, seed=77))
+def test_random_shapes_ring_f32(op, P, m, N, K, rings, order, variant, layout):
+    w = small(op, P, m, N, K, seed=P + m + N + K + 1, dist=0.1)
+    A_bits, B_bits = wl.make_inputs(w)
+    pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, rings=rings, rs_variant=api.RS_RING_RMW_F32, b_layout=layout)
+    A = [api.to_device(a) for a in A_bits]
+    B = [api.to_device(np.ascontiguousarray(b.T) if layout == api.B_KN else b) for b in B_bits]
+    outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    ws = api.alloc_workspace(pr)
+    api.compass_gemm_rs(pr, A, B, [o.view for o in outs], ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    assert all(o.guards_intact() for o in outs)
+    check_all([o.bits() for o in outs], ops.gemm_rs(A_bits, B_bits, rings=rings), w.name)
 
 
 @pytest.mark.parametrize("op,P,m,N,K,rings,order,variant,layout", _random_cases(40, seed=20261125))
