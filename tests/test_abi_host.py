@@ -254,6 +254,12 @@ def test_workspace_sizes():
     ring = api.make_problem(OP_GEMM_RS, 8, 8192, 4096, 1376, rs_variant=api.RS_RING_RMW)
     code, n = _codes(ring)
     assert code == api.OK and n >= api.STATUS_BYTES + 16 * 4 * 16 * 4
+    # the same with the running sum in FP32 scratch: the counters plus P owners x [M/P x N] floats
+    ring32 = api.make_problem(OP_GEMM_RS, 8, 8192, 4096, 1376, rs_variant=api.RS_RING_RMW_F32)
+    assert _codes(ring32) == (api.OK, n + 8 * 1024 * 4096 * 4)
+    assert _codes(api.make_problem(OP_GEMM_RS, 8, 8192, 4096, 1376, rs_variant=3))[0] == api.ERR_INVALID_ARG
+    plan32 = api.compass_launch_plan(ring32)
+    assert [(b.rank, b.step, b.ring) for b in plan32] == [(b.rank, b.step, b.ring) for b in api.compass_launch_plan(ring)]
 
 
 def test_fused_calls_refuse_bad_arguments_before_touching_the_gpu():
