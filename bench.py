@@ -276,6 +276,45 @@ def timing_protocol_report(torch, api, ops_by_name):
     return out
 
 
+def rs_variants_report(torch, api, op):
+    """The three GEMM+ReduceScatter forms on the benchmark's GEMM-RS shape, on the device buffers of the timed step:
+    segmented K (the reduction is the accumulator), ring read-modify-write with the running sum in the BF16 output
+    rows, and with the running sum in FP32 scratch.  The three are timed in turn inside one loop (30 rounds, a
+    synchronisation after every launch, after a pause that lets the board recover from the sustained loops before it),
+    so they are compared at the same board state."""
+    stream = torch.cuda.current_stream()
+    w = op.w
+    runs = {}
+    for name, variant in (("segmented_k", api.RS_SEGMENTED_K), ("ring_rmw", api.RS_RING_RMW), ("ring_rmw_f32", api.RS_RING_RMW_F32)):
+        pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, rs_variant=variant)
+        ws = api.alloc_workspace(pr)
+        runs[name] = (pr, ws)
+    call = lambda name: api.compass_gemm_rs(runs[name][0], op.A, op.B, op.out, runs[name][1], stream)
+    for _ in range(3):
+        for name in runs:
+            call(name)
+    torch.cuda.synchronize()
+    time.sleep(1.5)
+    ts = {name: [] for name in runs}
+    for _ in range(30):
+        for name in runs:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            call(name)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ts[name].append(e0.elapsed_time(e1))
+    out = {"workload": w.name, "timing": "median of 30 rounds; every round times each variant once, in turn"}
+    for name, (pr, ws) in runs.items():
+        status = api.compass_read_status(ws)
+        if status != (api.OK, 0):
+            raise SystemExit(f"device-side status of GEMM+ReduceScatter variant {name}: {status}")
+        med = float(np.median(ts[name]))
+        out[name] = {"ms_median": med, "tflops": w.flops / (med * 1e-3) / 1e12,
+                     "frac_of_nominal_2250": w.flops / (med * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS}
+    return out
+
+
 def mlp_report(torch, api):
     """The chained MLP block (Section II-A: AllGather -> GEMM0 -> GEMM1 -> ReduceScatter) on the 7B shape:
     two fused kernels back to back through compass_mlp_block, SwiGLU applied in the first kernel's epilogue."""
@@ -743,6 +782,7 @@ def run_ours(args, w_ag, w_rs):
         }
         if protocol is not None:
             line["timing_protocol"] = protocol
+            line["gemm_rs_variants"] = rs_variants_report(torch, api, rs)
             line["mlp_block"] = mlp_report(torch, api)
             torch.cuda.empty_cache()
             line["interdecom"] = interdecom_report(torch, api, peaks["hbm_gbs"], args.recalibrate)

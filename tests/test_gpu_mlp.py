@@ -87,6 +87,18 @@ def test_mlp_block_with_ring_rmw_reduction(act):
         assert rep.violations == 0 and rep.rms_rel <= np.sqrt(4) * 2.0 ** -9, f"rank {r}: {rep}"
 
 
+def test_mlp_block_with_ring_reduction_in_fp32_scratch():
+    """The block's second kernel as the ring read-modify-write with the running sum in FP32 scratch (the block's
+    workspace holds it): the single-rounding limits apply."""
+    act = omlp.ACT_SWIGLU
+    X, W0, W1, hc = make_inputs(4, 512, 256, 768, act)
+    H_gpu, Out_gpu = run_block(4, 512, 256, 768, act, X, W0, W1, hc, rs_variant=api.RS_RING_RMW_F32)
+    Out_ref, _ = omlp.mlp_block(X, W0, W1, act)
+    for r in range(4):
+        rep = compare.check(Out_gpu[r], Out_ref[r])
+        assert rep.ok, f"rank {r}: {rep}"
+
+
 def test_activation_special_values():
     """Accumulator values that stress the activations: zero and large magnitudes of either sign."""
     P, m, hidden, ffn = 1, 128, 16, 256
