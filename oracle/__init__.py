@@ -13,6 +13,8 @@ operators  AllGather+GEMM, GEMM+ReduceScatter, InterDecom(d) in FP64
 models     Eq. 2-5 (decomposition model, optimal degree), Eq. 7-8 (fusion
            model), Algorithm 1 (strategy selector), calibration regressions
 compare    the acceptance rule |gpu - ref| <= 1e-2 * max|ref| + 1e-3
+mlp        the tensor-parallel MLP block of Section II-A (both collectives through
+           ``operators``, activation in FP64, one rounding of the intermediate)
 
 Pins (what each part is checked against, other than itself) live in
 ``tests/test_oracle_*.py``.  Parts whose *numerical agreement with the paper's
