@@ -77,9 +77,14 @@ enum { COMPASS_DTYPE_BF16 = 0 };
  *     schedule order and added into the owner's rows in ring order by a
  *     vectorised read-modify-write in the GEMM epilogue.  The running sum lives
  *     in the BF16 output rows (what a BF16 ring transfer would carry), so the
- *     result is rounded once per contributor (the per-element error grows
- *     like sqrt(P): within 1e-2 * max|result| + 1e-3 for P <= 8, exceeded by
- *     rare elements at P = 16); the owner's contribution, scheduled last,
+ *     result is rounded once per contributor: it equals, on more than 99 % of
+ *     the elements bit for bit, the ring reduce-scatter computed hop by hop
+ *     with BF16 messages in the table's order.  Against the exact sum the
+ *     error grows like sqrt(P) roundings: RMS within sqrt(P) * 2^-9, and the
+ *     bound 1e-2 * max|result| + 1e-3 is met by all but about one element in
+ *     1e7..1e8 at P = 8 (a few in 1e6 at P = 16), which exceed it by a few per
+ *     cent.  Where that bound must hold on every element use SEGMENTED_K or
+ *     RING_RMW_F32.  The owner's contribution, scheduled last,
  *     completes it.  Needs one int32 counter per output tile in
  *     the workspace (zero before the first call; every call leaves them zero,
  *     unless it reported COMPASS_ERR_TIMEOUT: then re-initialise the workspace). */

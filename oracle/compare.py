@@ -7,6 +7,11 @@ GPU side is a violation.  Because the bound is loose, the comparison also
 reports the RMS error relative to the RMS of the reference and the fraction of
 elements within one BF16 ulp of the correctly rounded reference; the tests
 additionally require ``rms_rel <= 2**-8``.
+
+A reduce-scatter ring whose messages are BF16 rounds its running sum once per
+contributor; ``check_bf16_ring`` holds such a result against the hop-by-hop
+reference (``operators.gemm_rs(..., bf16_hops=True)``) and, with limits that
+account for the P roundings, against the exact sum.
 """
 from __future__ import annotations
 
@@ -61,3 +66,47 @@ def check(gpu_bits: np.ndarray, ref: np.ndarray, max_ref: float | None = None) -
     return Report(ok=(violations == 0 and rms_rel <= RMS_REL_LIMIT), violations=violations,
                   max_abs_err=max_err, tol=tol, max_ref=mref, rms_rel=rms_rel,
                   frac_within_1ulp=within, worst_index=tuple(int(i) for i in worst))
+
+
+@dataclass
+class RingReport:
+    ok: bool
+    identical: float            # fraction of elements equal to the hop-by-hop reference, bit for bit
+    min_identical: float
+    hops: Report                # against the hop-by-hop reference (tolerance from max|exact|)
+    exact: Report               # against the exact sum
+    allowed_beyond_bound: int
+
+    def __str__(self) -> str:
+        return (f"ok={self.ok} identical={self.identical:.5f} (>= {self.min_identical:.5f}) | vs hops: {self.hops} | "
+                f"vs exact (<= {self.allowed_beyond_bound} beyond the bound): {self.exact}")
+
+
+def check_bf16_ring(gpu_bits: np.ndarray, exact: np.ndarray, hops: np.ndarray, P: int, K: int,
+                    max_ref: float | None = None) -> RingReport:
+    """A GEMM+ReduceScatter result whose running sum was rounded to BF16 after every contributor.
+
+    Against ``hops`` (the same ring computed hop by hop in the schedule's order, every hop's addition in FP32 and its
+    rounding to BF16, partial products exact): the roundings are the same decisions on both sides except where the
+    GPU's FP32 accumulation of a K-term partial falls on the other side of a rounding boundary than the exact partial.
+    That happens to a fraction of about 1e-6 * K of the elements (a relative accumulation error of some K * 2^-24
+    against rounding intervals of 2^-8); a different ORDER of the contributors changes a quarter of the elements.
+    Required: at least 1 - max(1e-3, 3e-6 * K) of the elements identical, every element within the acceptance
+    bound, RMS difference at most 2^-11 of the RMS of the result.
+
+    Against ``exact``: P roundings of up to 2^-8 relative each (RMS about 2^-9.3 each) cannot promise
+    1e-2 * max|ref| on every element -- the worst case is P * 2^-8 -- and do not: at P = 8 about one element in
+    1e7..1e8, among the largest of its tensor, lands a few per cent beyond the bound, at P = 16 a few in 1e6.
+    Required: RMS error at most sqrt(P) * 2^-9 (2^-8 at least), no error beyond twice the bound, and at most
+    1e-6 (P <= 8) or 1e-4 (P > 8) of the elements, rounded up, beyond the bound."""
+    mref = float(np.max(np.abs(exact))) if max_ref is None else float(max_ref)
+    against_hops = check(gpu_bits, hops, max_ref=mref)
+    against_exact = check(gpu_bits, exact, max_ref=mref)
+    identical = float(np.mean(bf16_bits_to_f64(gpu_bits) == hops)) if hops.size else 1.0
+    min_identical = 1.0 - max(1e-3, 3e-6 * K)
+    allowed = int(np.ceil((1e-6 if P <= 8 else 1e-4) * exact.size))
+    ok = (identical >= min_identical and against_hops.violations == 0 and against_hops.rms_rel <= 2.0 ** -11
+          and against_exact.rms_rel <= max(RMS_REL_LIMIT, 2.0 ** -9 * P ** 0.5)
+          and against_exact.max_abs_err <= 2.0 * against_exact.tol and against_exact.violations <= allowed)
+    return RingReport(ok=ok, identical=identical, min_identical=min_identical, hops=against_hops,
+                      exact=against_exact, allowed_beyond_bound=allowed)

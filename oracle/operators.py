@@ -45,6 +45,28 @@ def f64_to_bf16_f64(x: np.ndarray) -> np.ndarray:
     return u.view(np.float32).astype(np.float64)
 
 
+def fp32_to_bf16_rne(x: np.ndarray) -> np.ndarray:
+    """Round FP32 values to the nearest BF16, ties to even (exact: one rounding
+    of a binary32 value); result as FP64."""
+    assert x.dtype == np.float32
+    u = x.view(np.uint32)
+    u = (u + (((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF))) & np.uint32(0xFFFF0000)
+    return u.view(np.float32).astype(np.float64)
+
+
+def hop_in_bf16(running: np.ndarray, partial: np.ndarray) -> np.ndarray:
+    """One hop of a reduce-scatter ring whose messages have the output's type,
+    BF16 (Section III-B: a rank adds its partial to the sum it received and
+    sends the result on; the paper does not state the type of the message, this
+    is the reading in which the ring moves tensors of the operator's own type).
+    The arriving sum is a BF16 value, the rank's own partial an FP32
+    accumulator; they are added in FP32 and the sum is rounded to BF16 for the
+    next message.  This decides a rounding, so it is taken in that precision
+    and not in FP64."""
+    s = running.astype(np.float32) + partial.astype(np.float32)
+    return fp32_to_bf16_rne(s)
+
+
 def gather_in_schedule_order(A: Sequence[np.ndarray], table: np.ndarray, rank: int) -> np.ndarray:
     """Rank `rank`'s private gather buffer, filled partition by partition in
     the order of its schedule entries.  Every row must be written exactly once."""
@@ -86,12 +108,17 @@ def ag_gemm(A: Sequence[np.ndarray], B: Sequence[np.ndarray], table: Optional[np
 
 
 def gemm_rs(A: Sequence[np.ndarray], B: Sequence[np.ndarray], table: Optional[np.ndarray] = None,
-            rings: int = 2, chunks: Optional[Sequence[int]] = None) -> List[np.ndarray]:
+            rings: int = 2, chunks: Optional[Sequence[int]] = None, bf16_hops: bool = False) -> List[np.ndarray]:
     """Out_c = rows [c*m,(c+1)*m) of sum_q A_q * B_q, reduced along the ring.
 
     For every partition the running sum starts at the rank whose table lists
     that partition at step 0 and visits the ranks in step order; the last
-    contributor must be the owner (Section III-B: local partition last)."""
+    contributor must be the owner (Section III-B: local partition last).
+
+    ``bf16_hops=False``: the sum itself (FP64), whatever the ring carries.
+    ``bf16_hops=True``: the result of a ring whose messages are BF16 -- the sum
+    is rounded once per contributor (``hop_in_bf16``), so the result depends on
+    the ORDER of the contributors; the values returned are BF16 values."""
     P = len(A)
     M, K = A[0].shape
     N = B[0].shape[0]
@@ -115,7 +142,8 @@ def gemm_rs(A: Sequence[np.ndarray], B: Sequence[np.ndarray], table: Optional[np
         for e in entries:
             assert int(e[ROW_BEGIN]) == rb and int(e[ROW_COUNT]) == rc and int(e[CHUNK]) == c
             q = int(e[RANK])
-            running += bf16_bits_to_f64(A[q][rb:rb + rc]) @ Bf[q].T
+            partial = bf16_bits_to_f64(A[q][rb:rb + rc]) @ Bf[q].T
+            running = hop_in_bf16(running, partial) if bf16_hops else running + partial
         assert int(entries[-1][RANK]) == c, "the running sum must end at the owner"
         if c not in out:
             out[c] = np.full((m, N), np.nan)
@@ -129,7 +157,7 @@ def gemm_rs(A: Sequence[np.ndarray], B: Sequence[np.ndarray], table: Optional[np
 
 
 def gemm_rs_rows(A: Sequence[np.ndarray], B: Sequence[np.ndarray], rows: np.ndarray,
-                 table: Optional[np.ndarray] = None, rings: int = 2):
+                 table: Optional[np.ndarray] = None, rings: int = 2, bf16_hops: bool = False):
     """GEMM+ReduceScatter restricted to some rows of the reduced [M x N] tensor
     (sorted global row indices), for sampling large cases.  Same ring order as
     ``gemm_rs``.  Returns {owner chunk: (rows inside the owner's block, values)}."""
@@ -153,7 +181,8 @@ def gemm_rs_rows(A: Sequence[np.ndarray], B: Sequence[np.ndarray], rows: np.ndar
         running = np.zeros((sel.size, Bf[0].shape[0]))
         for e in entries:
             q = int(e[RANK])
-            running += bf16_bits_to_f64(A[q][sel]) @ Bf[q].T
+            partial = bf16_bits_to_f64(A[q][sel]) @ Bf[q].T
+            running = hop_in_bf16(running, partial) if bf16_hops else running + partial
         assert int(entries[-1][RANK]) == c
         found.setdefault(c, []).append((sel - c * m, running))
     return {c: (np.concatenate([x[0] for x in v]), np.concatenate([x[1] for x in v])) for c, v in found.items()}

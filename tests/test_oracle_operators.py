@@ -200,3 +200,104 @@ def test_sampled_reduce_scatter_rows_equal_full_rows():
         assert np.array_equal(vals, full[c][local])
         seen += len(local)
     assert seen == len(rows)
+
+
+# ---- the ring with BF16 messages: one rounding per contributor, so the ORDER of the contributors shows ----------
+
+def scalar_shards(P, m, values):
+    """K = 1, N = 1, every weight 1.0: partial of rank q for row i is values[q][i] itself."""
+    A = [wl.f32_to_bf16_bits(np.asarray(values[q], dtype=np.float32).reshape(P * m, 1)) for q in range(P)]
+    B = [wl.f32_to_bf16_bits(np.ones((1, 1), dtype=np.float32)) for _ in range(P)]
+    return A, B
+
+
+def test_fp32_to_bf16_rounding_matches_torch_and_ties_go_to_even():
+    x = (np.random.default_rng(5).standard_normal(20000) * 41.0).astype(np.float32)
+    x[:6] = [257.0, 259.0, 261.0, -257.0, 1.00390625, 1.01171875]                 # exact ties
+    want = torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy()
+    got = ops.fp32_to_bf16_rne(x)
+    assert np.array_equal(got, want)
+    assert list(got[:4]) == [256.0, 260.0, 260.0, -256.0]                         # 8 significant bits: step 2 above 256
+
+
+def test_bf16_hops_single_ring_order_is_owner_plus_one_first_owner_last():
+    """Forward ring, P = 3, one row per chunk: the sum for chunk c starts at rank c+1 and ends at its owner c.
+    256 + 1 is a tie and rounds to 256 (even), twice; 1 + 1 + 256 = 258 is exact.  So where the large term comes
+    first the result is 256, where it comes last 258."""
+    P = 3
+    values = np.zeros((P, P))
+    values[1][0], values[2][0], values[0][0] = 256.0, 1.0, 1.0      # chunk 0: ranks 1, 2, 0
+    values[2][1], values[0][1], values[1][1] = 1.0, 1.0, 256.0      # chunk 1: ranks 2, 0, 1
+    values[0][2], values[1][2], values[2][2] = 256.0, 3.0, 1.0      # chunk 2: ranks 0, 1, 2: 259 -> 260, 261 -> 260
+    A, B = scalar_shards(P, 1, values)
+    out = ops.gemm_rs(A, B, rings=1, bf16_hops=True)
+    assert [float(o[0, 0]) for o in out] == [256.0, 258.0, 260.0]
+    exact = ops.gemm_rs(A, B, rings=1)
+    assert [float(o[0, 0]) for o in exact] == [258.0, 258.0, 260.0]
+
+
+def test_bf16_hops_double_ring_halves_travel_in_opposite_directions():
+    """P = 4, two rows per chunk.  Chunk 0's first row rides the backward ring (ranks 3, 2, 1, then the owner 0), its
+    second row the forward ring (ranks 1, 2, 3, 0).  With rank 1 holding 256 and ranks 2, 3 holding 1:
+    backward 1 + 1 = 2, + 256 = 258; forward 256 + 1 -> 256, + 1 -> 256."""
+    P, m = 4, 2
+    values = np.zeros((P, P * m))
+    for row in (0, 1):
+        values[1][row], values[2][row], values[3][row] = 256.0, 1.0, 1.0
+    A, B = scalar_shards(P, m, values)
+    out = ops.gemm_rs(A, B, rings=2, bf16_hops=True)
+    assert float(out[0][0, 0]) == 258.0 and float(out[0][1, 0]) == 256.0
+    sampled = ops.gemm_rs_rows(A, B, np.array([0, 1]), rings=2, bf16_hops=True)
+    assert list(sampled[0][1][:, 0]) == [258.0, 256.0]
+
+
+def test_bf16_hops_change_nothing_when_every_running_sum_is_a_bf16_value():
+    w = wl.Workload("ints", OP_GEMM_RS, P=4, M=32, N=8, K=16)
+    A, B = wl.make_structured_inputs(w, "index")
+    exact = ops.gemm_rs(A, B)
+    assert max(float(np.max(np.abs(e))) for e in exact) <= 256.0          # integers up to 256 are BF16 values
+    for got, want in zip(ops.gemm_rs(A, B, bf16_hops=True), exact):
+        assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("P", [1, 2, 5, 8])
+def test_bf16_hops_error_bound(P):
+    """Each hop rounds to nearest: at most half a BF16 step (8 significant bits: 2^-8 relative) of the sum after that
+    hop, plus the FP32 rounding of the addition.  P = 1 is the correctly rounded product."""
+    w, A, B = tiny(OP_GEMM_RS, P, P * 8, 16, 24, seed=11)
+    exact = ops.gemm_rs(A, B)
+    got = ops.gemm_rs(A, B, bf16_hops=True)
+    prefix_max = np.zeros_like(np.concatenate(exact))
+    table = schedule(OP_GEMM_RS, P, 2, w.M)
+    Bf = [ops.bf16_bits_to_f64(b) for b in B]
+    partial = [ops.bf16_bits_to_f64(A[q]) @ Bf[q].T for q in range(P)]
+    for row in range(w.M):                                            # largest |prefix sum| along the row's ring
+        order = [int(e[0]) for e in sorted((e for e in table if e[6] <= row < e[6] + e[7]), key=lambda e: int(e[1]))]
+        run = np.zeros(w.N)
+        for q in order:
+            run = run + partial[q][row]
+            prefix_max[row] = np.maximum(prefix_max[row], np.abs(run))
+    err = np.abs(np.concatenate(got) - np.concatenate(exact))
+    assert (err <= P * (2.0 ** -8 + 2.0 ** -23) * prefix_max * (1 + P * 2.0 ** -8)).all()
+    if P == 1:
+        want = torch.from_numpy(exact[0].astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+        assert np.array_equal(got[0], want)
+    else:
+        assert any(not np.array_equal(g, ops.f64_to_bf16_f64(e)) for g, e in zip(got, exact))   # the hops do show
+
+
+def test_rule_for_a_bf16_ring_tells_the_order_of_the_contributors():
+    """The hop-by-hop ring passes its own rule; the same sum reduced in the single ring's order (every partition
+    forward) or rounded once at the end is the right sum, within every tolerance against the exact result, and still
+    fails: too few elements are identical."""
+    w, A, B = tiny(OP_GEMM_RS, 8, 8 * 16, 24, 40, seed=7)
+    exact = ops.gemm_rs(A, B, rings=2)
+    hops = ops.gemm_rs(A, B, rings=2, bf16_hops=True)
+    other = ops.gemm_rs(A, B, rings=1, bf16_hops=True)
+    to_bits = lambda x: wl.f32_to_bf16_bits(x.astype(np.float32))
+    for c in range(8):
+        assert compare.check_bf16_ring(to_bits(hops[c]), exact[c], hops[c], 8, 40).ok
+        wrong = compare.check_bf16_ring(to_bits(other[c]), exact[c], hops[c], 8, 40)
+        assert not wrong.ok and wrong.identical < 0.95 and wrong.exact.violations == 0
+        once = compare.check_bf16_ring(to_bits(exact[c]), exact[c], hops[c], 8, 40)
+        assert not once.ok and once.exact.ok
