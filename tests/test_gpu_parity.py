@@ -986,6 +986,56 @@ def test_random_shapes_and_options(op, P, m, N, K, rings, order, variant, layout
     check_all([o.bits() for o in outs], refs, w.name)
 
 
+def _random_pipeline_cases(n, seed):
+    """InterDecom and push: degree, copy route, one or two streams and the weight layout drawn at random."""
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < n:
+        op = int(rng.integers(0, 2))
+        P = int(rng.choice([1, 2, 3, 4, 5, 8, 16]))
+        m = int(rng.choice([16, 48, 64, 128, 144, 256, 320, 512, 1024]))
+        N = int(rng.choice([8, 64, 136, 256, 264, 520, 776, 1032]))
+        K = int(rng.choice([8, 72, 128, 200, 344, 456, 1024]))
+        if P * P * m * N * K > 3e10:
+            continue
+        d = int(rng.choice([d for d in (1, 2, 4, 8, 16) if m % d == 0]))
+        cases.append((op, P, m, N, K, d, int(rng.integers(0, 2)), int(rng.integers(0, 2)), int(rng.integers(0, 2))))
+    return cases
+
+
+@pytest.mark.parametrize("op,P,m,N,K,d,layout,copy_mode,two_streams", _random_pipeline_cases(24, seed=31))
+def test_random_interdecom_and_push(op, P, m, N, K, d, layout, copy_mode, two_streams):
+    """Two calls on one workspace each: the second finds the flags, counters and staging buffers the first left."""
+    w = small(op, P, m, N, K, seed=P + m + N + K + d, dist=0.1)
+    A_bits, B_bits = wl.make_inputs(w)
+    refs = ops.ag_gemm(A_bits, B_bits) if op == wl.OP_AG_GEMM else ops.gemm_rs(A_bits, B_bits)
+    A = [api.to_device(a) for a in A_bits]
+    B = [api.to_device(np.ascontiguousarray(b.T) if layout == api.B_KN else b) for b in B_bits]
+    side = torch.cuda.Stream()
+    pr = api.make_problem(op, P, w.M, N, K, d=d, copy_mode=copy_mode, b_layout=layout)
+    ws = api.alloc_workspace(pr, api.WS_DECOMP)
+    torch.cuda.synchronize()
+    for call in range(2):
+        outs = [gu.Guarded(*w.out_shape) for _ in range(P)]
+        api.compass_decomp(pr, A, B, [o.view for o in outs], ws, torch.cuda.current_stream(), side if two_streams else None)
+        status = api.compass_read_status(ws)
+        torch.cuda.synchronize()
+        assert status == (api.OK, 0) and all(o.guards_intact() for o in outs)
+        check_all([o.bits() for o in outs], refs, f"{w.name} InterDecom d={d} call {call}")
+    if op != wl.OP_AG_GEMM:
+        return
+    pr = api.make_problem(op, P, w.M, N, K, b_layout=layout, order=copy_mode)
+    ws = api.alloc_workspace(pr, api.WS_PUSH)
+    torch.cuda.synchronize()
+    for call in range(2):
+        outs = [gu.Guarded(*w.out_shape) for _ in range(P)]
+        api.compass_ag_gemm_push(pr, A, B, [o.view for o in outs], ws, torch.cuda.current_stream(), side)
+        status = api.compass_read_status(ws)
+        torch.cuda.synchronize()
+        assert status == (api.OK, 0) and all(o.guards_intact() for o in outs)
+        check_all([o.bits() for o in outs], refs, f"{w.name} push call {call}")
+
+
 # ---- CUDA graphs -------------------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("which", ["fused_ag", "fused_rs_rmw", "decomp", "push", "mlp"])
