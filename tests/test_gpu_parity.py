@@ -1036,6 +1036,97 @@ def test_random_interdecom_and_push(op, P, m, N, K, d, layout, copy_mode, two_st
         check_all([o.bits() for o in outs], refs, f"{w.name} push call {call}")
 
 
+# ---- tensors beyond 4 GiB: 64-bit addressing on every path --------------------------------------------------------
+
+def _tiled(bits, rows):
+    """`rows` rows made of repetitions of a seeded block (cheap to generate; the period is not a power of two, so
+    an offset that wrapped at 2^31 or 2^32 lands on a different row)."""
+    reps = -(-rows // bits.shape[0])
+    return np.ascontiguousarray(np.tile(bits, (reps, 1))[:rows])
+
+
+def _run_large(op, P, m, N, K, variant, d, period=0):
+    """Outputs start as NaN; returns (inputs, outputs on the device, status)."""
+    w = wl.Workload("large", op, P=P, M=P * m, N=N, K=K, b_dist=("normal", 0.1), seed=5)
+    if period:
+        block = wl.Workload("block", op, P=P, M=P * period, N=min(N, period), K=K, b_dist=("normal", 0.1), seed=5)
+        A_small, B_small = wl.make_inputs(block)
+        A_bits = [_tiled(a, w.a_shape[0]) for a in A_small]
+        B_bits = [_tiled(b, N) for b in B_small]
+    else:
+        A_bits, B_bits = wl.make_inputs(w)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    outs = [torch.full(w.out_shape, float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(P)]
+    pr = api.make_problem(op, P, w.M, N, K, rs_variant=variant, d=max(d, 1))
+    if d:
+        ws = api.alloc_workspace(pr, api.WS_DECOMP)
+        side = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        api.compass_decomp(pr, A, B, outs, ws, torch.cuda.current_stream(), side)
+    else:
+        ws = api.alloc_workspace(pr)
+        (api.compass_ag_gemm if op == wl.OP_AG_GEMM else api.compass_gemm_rs)(pr, A, B, outs, ws)
+    status = api.compass_read_status(ws)
+    torch.cuda.synchronize()
+    return w, A_bits, B_bits, outs, status
+
+
+def _check_large(w, A_bits, B_bits, outs, status, byte_pitch, extra_rows=()):
+    """Every element written (no NaN left), and the rows at which a byte offset of `byte_pitch` per row passes
+    2^31, 2^32 and 2^33, the first and last rows and a random sample equal to the oracle's."""
+    assert status == (api.OK, 0)
+    assert all(int(torch.isnan(o).sum().item()) == 0 for o in outs)
+    P, m = w.P, w.M // w.P
+    rows_out = w.out_shape[0]
+    rows = {0, 1, rows_out - 2, rows_out - 1} | set(np.random.default_rng(1).integers(0, rows_out, 24).tolist()) | set(extra_rows)
+    for offset in (2 ** 31, 2 ** 32, 2 ** 33):
+        r = offset // byte_pitch
+        rows |= {r - 1, r, r + 1}
+    rows = np.array(sorted(r for r in rows if 0 <= r < rows_out))
+    take = lambda t, idx: t[torch.as_tensor(idx, device="cuda")].view(torch.int16).cpu().numpy().view(np.uint16)
+    if w.op == wl.OP_AG_GEMM:
+        for r in range(P):
+            (ref,) = ops.ag_gemm(A_bits, B_bits, ranks=[r], rows=rows)
+            rep = compare.check(take(outs[r], rows), ref)
+            assert rep.ok, f"rank {r}: {rep}"
+    else:
+        found = ops.gemm_rs_rows(A_bits, B_bits, np.array(sorted(c * m + int(r) for c in range(P) for r in rows)))
+        assert sorted(found) == list(range(P))
+        for c, (local, ref) in found.items():
+            rep = compare.check(take(outs[c], local), ref)
+            assert rep.ok, f"chunk {c}: {rep}"
+
+
+@pytest.mark.parametrize("op,P,m,variant,d", [
+    (wl.OP_AG_GEMM, 1, 70000, 0, 0), (wl.OP_AG_GEMM, 2, 35000, 0, 0), (wl.OP_AG_GEMM, 2, 35000, 0, 2),
+    (wl.OP_GEMM_RS, 2, 70000, api.RS_SEGMENTED_K, 0), (wl.OP_GEMM_RS, 2, 70000, api.RS_RING_RMW, 0),
+    (wl.OP_GEMM_RS, 2, 70000, api.RS_RING_RMW_F32, 0), (wl.OP_GEMM_RS, 2, 70000, api.RS_SEGMENTED_K, 2),
+])
+def test_outputs_beyond_4_gib(op, P, m, variant, d):
+    """70000 x 32776 BF16 per rank (4.6 GB): row 32760 starts beyond 2^31 bytes, row 65520 beyond 2^32."""
+    N = 32776
+    w, A_bits, B_bits, outs, status = _run_large(op, P, m, N, 64, variant, d)
+    _check_large(w, A_bits, B_bits, outs, status, byte_pitch=2 * N)
+
+
+@pytest.mark.parametrize("op,P,m,N,variant,d", [
+    (wl.OP_AG_GEMM, 2, 35000, 8, 0, 0), (wl.OP_AG_GEMM, 2, 35000, 8, 0, 2), (wl.OP_GEMM_RS, 2, 35000, 8, 0, 0),
+    (wl.OP_GEMM_RS, 2, 35000, 8, 0, 2), (wl.OP_AG_GEMM, 2, 16, 70000, 0, 0),
+])
+def test_inputs_beyond_4_gib(op, P, m, N, variant, d):
+    """K = 32768: an activation shard of 35000 (or 70000) rows, or a weight shard of 70000 rows, is 2.3-4.6 GB;
+    row 32768 of either starts at 2^31 bytes, row 65536 at 2^32."""
+    K = 32768
+    w, A_bits, B_bits, outs, status = _run_large(op, P, m, N, K, variant, d, period=1000)
+    # Output rows that read the activation rows around 2^31 and 2^32 bytes: AllGather+GEMM, row 32768 of either shard
+    # (gathered rows 32768 and m + 32768); GEMM+ReduceScatter, rows 32768 and 65536 of the [M x K] shards (owner 0's
+    # row 32768, owner 1's row 65536 - m).  The weight rows beyond those offsets are output COLUMNS: whole rows are
+    # compared.
+    around = lambda r: {r - 1, r, r + 1}
+    extra = around(32768) | (around(m + 32768) if op == wl.OP_AG_GEMM else around(65536 - m))
+    _check_large(w, A_bits, B_bits, outs, status, byte_pitch=2 * N, extra_rows=extra)
+
+
 # ---- CUDA graphs -------------------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("which", ["fused_ag", "fused_rs_rmw", "decomp", "push", "mlp"])
