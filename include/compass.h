@@ -74,26 +74,29 @@ enum { COMPASS_DTYPE_BF16 = 0 };
  *     in ring order (the reduction tree is the tensor-core accumulator); one
  *     BF16 rounding.
  *   RING_RMW: every rank's partial tile is produced separately in that rank's
- *     schedule order and added into the owner's rows in ring order by a
- *     vectorised read-modify-write in the GEMM epilogue.  The running sum lives
- *     in the BF16 output rows (what a BF16 ring transfer would carry), so the
- *     result is rounded once per contributor: it equals, on more than 99 % of
+ *     schedule order and added to the partition's running sum in ring order by
+ *     the GEMM epilogue.  The running sum is BF16 (what a BF16 ring transfer
+ *     would carry) and travels from contributor to contributor through scratch
+ *     in the workspace; the owner's contribution, scheduled last, writes the
+ *     output rows (which never hold a partial sum).  The result is rounded once
+ *     per contributor: it equals, on more than 99 % of
  *     the elements bit for bit, the ring reduce-scatter computed hop by hop
  *     with BF16 messages in the table's order.  Against the exact sum the
  *     error grows like sqrt(P) roundings: RMS within sqrt(P) * 2^-9, and the
  *     bound 1e-2 * max|result| + 1e-3 is met by all but about one element in
  *     1e7..1e8 at P = 8 (a few in 1e6 at P = 16), which exceed it by a few per
  *     cent.  Where that bound must hold on every element use SEGMENTED_K or
- *     RING_RMW_F32.  The owner's contribution, scheduled last,
- *     completes it.  Needs one int32 counter per output tile in
- *     the workspace (zero before the first call; every call leaves them zero,
- *     unless it reported COMPASS_ERR_TIMEOUT: then re-initialise the workspace). */
+ *     RING_RMW_F32.  Needs, in the workspace, one int32 counter per 128 x 256
+ *     fragment of the output (zero before the first call; every call leaves
+ *     them zero, unless it reported COMPASS_ERR_TIMEOUT: then re-initialise the
+ *     workspace) and 64 KB of scratch per counter (about P * (M/P) * N * 2
+ *     bytes; never initialised, never read by the caller). */
 /*   RING_RMW_F32: the same ordered ring accumulation with the running sum kept
- *     in FP32 scratch inside the workspace (what an FP32 ring transfer would
- *     carry: twice the bytes per hop): contributors add their FP32 partial
- *     tile to it in ring order and the owner's contribution, last, writes the
- *     BF16 result -- one rounding, whatever P.  Needs the tile counters of
- *     RING_RMW plus P * (M/P) * N * 4 bytes in the workspace. */
+ *     in FP32 (what an FP32 ring transfer would carry: twice the bytes per
+ *     hop): contributors add their FP32 partial tile to it in ring order and
+ *     the owner's contribution, last, writes the BF16 result -- one rounding,
+ *     whatever P.  Needs the tile counters of RING_RMW and 128 KB of scratch
+ *     per counter (about P * (M/P) * N * 4 bytes). */
 enum { COMPASS_RS_SEGMENTED_K = 0, COMPASS_RS_RING_RMW = 1, COMPASS_RS_RING_RMW_F32 = 2 };
 enum { COMPASS_STRATEGY_INTRAFUSION = 0, COMPASS_STRATEGY_INTERDECOM = 1 };
 /* Launch order of the fused kernels.  Every rank's tiles are always issued in
@@ -243,7 +246,7 @@ int compass_ag_gemm_push(const compass_problem* problem, const void* const* A, c
  * is deadlock-free because all CTAs of the launch are resident at once, and
  * the grid is sized for an otherwise idle GPU.  Run nothing else on the GPU's
  * SMs for the duration of the call, and read compass_read_status after it: on
- * COMPASS_ERR_TIMEOUT the output holds partial sums and the tile counters are
+ * COMPASS_ERR_TIMEOUT the output is incomplete and the tile counters are
  * dirty (re-initialise the workspace).  The segmented-K variant has no such
  * waits. */
 int compass_gemm_rs(const compass_problem* problem, const void* const* A, const void* const* B,

@@ -224,13 +224,18 @@ int plan_fused(const compass_problem* pr, GemmLaunch* L, compass_plan_block* vie
   return COMPASS_OK;
 }
 
-// FP32 running sums of the ring read-modify-write variant with FP32 scratch: behind the tile counters, one per owner.
+// Running sums of the ring read-modify-write variants: behind the tile counters, one 128 x 256 fragment per counter
+// (BF16 or FP32), in the order the epilogue's lanes hold them.
+size_t ring_scratch_bytes(const compass_problem* pr) {
+  if (pr->op != COMPASS_OP_GEMM_RS || pr->rs_variant == COMPASS_RS_SEGMENTED_K) return 0;
+  const size_t element = pr->rs_variant == COMPASS_RS_RING_RMW_F32 ? sizeof(float) : 2;
+  return rmw_counter_count(pr) * size_t(BM) * size_t(BN) * element;
+}
+
 void set_running_sums(const compass_problem* pr, GemmLaunch* L, void* ws) {
-  for (int r = 0; r < kMaxP; ++r) L->sum_ptr[r] = nullptr;
-  if (pr->op != COMPASS_OP_GEMM_RS || pr->rs_variant != COMPASS_RS_RING_RMW_F32) return;
-  uint8_t* base = static_cast<uint8_t*>(ws) + COMPASS_STATUS_BYTES + align_up(rmw_counter_count(pr) * sizeof(int32_t));
-  const size_t per_owner = align_up(size_t(pr->M / pr->P) * size_t(pr->N) * sizeof(float));
-  for (int r = 0; r < pr->P; ++r) L->sum_ptr[r] = reinterpret_cast<float*>(base + size_t(r) * per_owner);
+  L->ring_scratch = nullptr;
+  if (ring_scratch_bytes(pr) == 0) return;
+  L->ring_scratch = static_cast<uint8_t*>(ws) + COMPASS_STATUS_BYTES + align_up(rmw_counter_count(pr) * sizeof(int32_t));
 }
 
 int fused_call(const compass_problem* pr, int op, const void* const* A, const void* const* B, void* const* out, void* ws,
@@ -479,8 +484,7 @@ extern "C" int compass_workspace_bytes(const compass_problem* pr, int which, siz
   if (which == COMPASS_WS_FUSED) {
     if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant != COMPASS_RS_SEGMENTED_K)
       total += align_up(rmw_counter_count(pr) * sizeof(int32_t));
-    if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant == COMPASS_RS_RING_RMW_F32)
-      total += size_t(pr->P) * align_up(size_t(pr->M / pr->P) * size_t(pr->N) * sizeof(float));
+    total += align_up(ring_scratch_bytes(pr));
   } else if (which == COMPASS_WS_DECOMP) {
     const size_t inner = pr->op == COMPASS_OP_AG_GEMM ? size_t(pr->K) : size_t(pr->N);
     total += size_t(pr->P) * align_up(size_t(pr->M) * inner * 2);

@@ -11,7 +11,8 @@
 //   GEMM+ReduceScatter, segmented K: the k-loop of a tile runs over the P ranks'
 //     K slices in ring order into one TMEM accumulator (in-kernel reduction);
 //   GEMM+ReduceScatter, ring read-modify-write: every rank's partial tile is
-//     added by the epilogue into the owner's rows in ring order.
+//     added by the epilogue to the partition's running sum in ring order (the
+//     sum travels through scratch memory; the owner, last, writes its rows).
 //
 // Three kernels share the roles and the barrier protocol:
 //   gemm_mixed_kernel  clusters of two CTAs; 512x256 tiles (two accumulators per
@@ -258,8 +259,8 @@ struct StageIter {
 };
 
 // kAct: the plain-store epilogue applies p.activation (its own instantiation, see gemm_mixed_kernel).
-// kF32Sum: the ring read-modify-write epilogue keeps the running sum in FP32 scratch (p.sum) and only the last
-// contributor writes the BF16 output (again its own instantiation).
+// kF32Sum: the ring read-modify-write epilogue keeps the running sum in FP32 instead of BF16 (again its own
+// instantiation).
 template <bool kPair, bool kAct, bool kF32Sum>
 __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
   using C = Cfg<kPair>;
@@ -498,23 +499,25 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
       const int npass = (ocols + 63) >> 6;
 
       if constexpr (kF32Sum) {
-        // Ring read-modify-write with the running sum in FP32 scratch.  Same counters and ordering as below; the
-        // sum travels as 32-column pieces (128 bytes per row: 4 rows per load or store instruction, transposed
-        // through shared memory into one row per lane), four pieces in flight ahead of the one being added.
+        // Ring read-modify-write with the running sum in FP32 scratch.  Same counters and ordering as below.  A
+        // fragment's sum lies in the scratch in the order the lanes hold it (64 groups of 4 columns per warp, each
+        // group the 32 lanes' 16 bytes in a row): a lane reads and writes its own row, every instruction of the
+        // warp moves 512 contiguous bytes, and nothing passes through shared memory, whose bandwidth the tensor
+        // core needs for its operands.  Four 32-column pieces are in flight ahead of the one being added.
         const bool live = frag.r0 < p.rows_per_block;          // a fragment past the block adds nothing
         const bool add_previous = live && b.step > 0;
         const bool last = int(b.step) == p.last_step;          // the owner's contribution: writes the BF16 result
-        int* counter = p.tile_counters + (int64_t(b.part) * p.frags_m + frag.r0 / BM) * p.tiles_n + tc.nt;
-        float* sbase = p.sum[b.out_idx] + int64_t(b.out_row0 + first_row) * p.N + int64_t(tc.nt) * BN;
+        const int64_t frag_idx = (int64_t(b.part) * p.frags_m + frag.r0 / BM) * p.tiles_n + tc.nt;
+        int* counter = p.tile_counters + frag_idx;
+        uint4* sfrag = reinterpret_cast<uint4*>(p.ring_scratch + frag_idx * int64_t(BM * BN * 4)) + quarter * (BN / 4) * 32 + lane;
+        const bool row_ok = first_row + lane < p.rows_per_block;
         uint4 ahead[4][8];
         auto fetch = [&](int piece, uint4 (&dst)[8]) {
-          const int col = piece * 32 + seg * 4;
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const int r = i * 4 + (lane >> 3);
+            const int g = piece * 8 + i;
             dst[i] = make_uint4(0u, 0u, 0u, 0u);
-            if (first_row + r < p.rows_per_block && col < ncols)
-              dst[i] = __ldcg(reinterpret_cast<const uint4*>(sbase + int64_t(r) * p.N + col));
+            if (row_ok && g * 4 < ncols) dst[i] = __ldcg(sfrag + g * 32);       // written by another SM: from L2
           }
         };
         if (add_previous) {
@@ -533,18 +536,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
           float prev[32];
           if (add_previous) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-              *reinterpret_cast<uint4*>(stage + (i * 4 + (lane >> 3)) * kStageRowBytes + seg * 16) = ahead[c & 3][i];
-            __syncwarp();
-#pragma unroll
-            for (int g = 0; g < 8; ++g) {
-              const uint4 q = *reinterpret_cast<const uint4*>(stage + lane * kStageRowBytes + g * 16);
-              prev[g * 4 + 0] = __uint_as_float(q.x);
-              prev[g * 4 + 1] = __uint_as_float(q.y);
-              prev[g * 4 + 2] = __uint_as_float(q.z);
-              prev[g * 4 + 3] = __uint_as_float(q.w);
+            for (int i = 0; i < 8; ++i) {
+              prev[i * 4 + 0] = __uint_as_float(ahead[c & 3][i].x);
+              prev[i * 4 + 1] = __uint_as_float(ahead[c & 3][i].y);
+              prev[i * 4 + 2] = __uint_as_float(ahead[c & 3][i].z);
+              prev[i * 4 + 3] = __uint_as_float(ahead[c & 3][i].w);
             }
-            __syncwarp();
             if (c + 4 < BN / 32) fetch(c + 4, ahead[c & 3]);
           }
           uint32_t v[32];
@@ -584,25 +581,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
               }
               __syncwarp();
             } else {
-              // FP32 running sum: 128 bytes per row; every store instruction writes 4 rows x 128 contiguous bytes
-              uint4* srow = reinterpret_cast<uint4*>(stage + lane * kStageRowBytes);
-#pragma unroll
-              for (int g = 0; g < 8; ++g) srow[g] = make_uint4(v[g * 4 + 0], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
-              __syncwarp();
-              const int col = c * 32 + seg * 4;
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                const int r = i * 4 + (lane >> 3);
-                if (first_row + r < p.rows_per_block && col < ncols)
-                  *reinterpret_cast<uint4*>(sbase + int64_t(r) * p.N + col) =
-                      *reinterpret_cast<const uint4*>(stage + r * kStageRowBytes + seg * 16);
+                const int g = c * 8 + i;
+                if (row_ok && g * 4 < ncols) sfrag[g * 32] = make_uint4(v[i * 4 + 0], v[i * 4 + 1], v[i * 4 + 2], v[i * 4 + 3]);
               }
-              __syncwarp();
             }
           }
         }
         if (live) {
-          // the warp barriers above ordered every lane's stores before lane 0's release of the counter
+          // the warp barrier orders every lane's stores before lane 0's release of the counter
+          __syncwarp();
           if (lane == 0) {
             int before;
             asm volatile("atom.add.release.gpu.global.s32 %0, [%1], 1;" : "=r"(before) : "l"(counter) : "memory");
@@ -615,17 +604,27 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 
       // Ring read-modify-write: contributor `step` of a partition adds its
       // partial tile to the running sum that contributor step-1 left in the
-      // owner's rows.  One counter per 128 x 256 fragment of the output counts
+      // scratch, and passes the sum on there; the owner, last, writes it to its
+      // rows instead.  One counter per 128 x 256 fragment of the output counts
       // the epilogue warps that have finished; contributor s starts when all
       // four warps of s-1 have.  (Per fragment, not per tile: the two CTAs of a
       // pair may be working on different partitions.)
       const bool rmw = p.epilogue == EPI_RING_RMW && frag.r0 < p.rows_per_block;   // a fragment past the block adds nothing
       const bool add_previous = rmw && b.step > 0;
+      const bool pass_on = rmw && int(b.step) != p.last_step;    // not the owner's contribution: the sum goes to the scratch
       int* counter = nullptr;
+      // The fragment's running sum lies in the scratch in the order the lanes hold it: 32 groups of 8 columns per
+      // warp, each group the 32 lanes' 16 bytes in a row.  A lane reads and writes its own row, every instruction
+      // of the warp moves 512 contiguous bytes, and nothing passes through shared memory, whose bandwidth the
+      // tensor core needs for its operands.
+      uint4* sfrag = nullptr;
+      const bool row_ok = first_row + lane < p.rows_per_block;
       // `sum` first holds this lane's row of the running sum (packed BF16 pairs), then the row to store.
       uint32_t sum[BN / 2];
       if (rmw) {
-        counter = p.tile_counters + (int64_t(b.part) * p.frags_m + frag.r0 / BM) * p.tiles_n + tc.nt;
+        const int64_t frag_idx = (int64_t(b.part) * p.frags_m + frag.r0 / BM) * p.tiles_n + tc.nt;
+        counter = p.tile_counters + frag_idx;
+        sfrag = reinterpret_cast<uint4*>(p.ring_scratch + frag_idx * int64_t(BM * BN * 2)) + quarter * (BN / 8) * 32 + lane;
         if (add_previous) {
           // All of this happens while the tile's MMAs are still running: the wait for the previous
           // contributor and the fetch of its running sum need nothing from the accumulator.
@@ -635,43 +634,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
           // lane 0 acquired the counter; the warp barrier orders the other lanes' loads of the running sum behind it
           __syncwarp();
           if (!ready) break;
-          // The warp's 32 rows x 256 columns come in as whole 128-byte row pieces (4 rows per load instruction,
-          // every sector fully used), all 32 loads of a lane in flight at once, and are then transposed through
-          // shared memory, 64 columns at a time, into one row per lane (in place in `sum`).
+          // all 32 loads of a lane in flight at once
 #pragma unroll
-          for (int pass = 0; pass < BN / 64; ++pass) {
-            const int col = pass * 64 + seg * 8;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const int r = i * 4 + (lane >> 3);
-              uint4 piece = make_uint4(0u, 0u, 0u, 0u);
-              if (pass < npass && first_row + r < p.rows_per_block && col < ocols)
-                piece = __ldcg(reinterpret_cast<const uint4*>(obase + int64_t(r) * p.ldo + col));   // written by another SM: from L2
-              sum[pass * 32 + i * 4 + 0] = piece.x;
-              sum[pass * 32 + i * 4 + 1] = piece.y;
-              sum[pass * 32 + i * 4 + 2] = piece.z;
-              sum[pass * 32 + i * 4 + 3] = piece.w;
-            }
-          }
-#pragma unroll
-          for (int pass = 0; pass < BN / 64; ++pass) {
-            if (pass < npass) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                *reinterpret_cast<uint4*>(stage + (i * 4 + (lane >> 3)) * kStageRowBytes + seg * 16) =
-                    make_uint4(sum[pass * 32 + i * 4 + 0], sum[pass * 32 + i * 4 + 1], sum[pass * 32 + i * 4 + 2],
-                               sum[pass * 32 + i * 4 + 3]);
-              __syncwarp();
-#pragma unroll
-              for (int g = 0; g < 8; ++g) {
-                const uint4 q = *reinterpret_cast<const uint4*>(stage + lane * kStageRowBytes + g * 16);
-                sum[pass * 32 + g * 4 + 0] = q.x;
-                sum[pass * 32 + g * 4 + 1] = q.y;
-                sum[pass * 32 + g * 4 + 2] = q.z;
-                sum[pass * 32 + g * 4 + 3] = q.w;
-              }
-              __syncwarp();
-            }
+          for (int g = 0; g < BN / 8; ++g) {
+            uint4 piece = make_uint4(0u, 0u, 0u, 0u);
+            if (row_ok && g * 8 < ncols) piece = __ldcg(sfrag + g * 32);          // written by another SM: from L2
+            sum[g * 4 + 0] = piece.x;
+            sum[g * 4 + 1] = piece.y;
+            sum[g * 4 + 2] = piece.z;
+            sum[g * 4 + 3] = piece.w;
           }
         }
       }
@@ -715,11 +686,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         if (kPair) mbar_arrive_cluster(map_to_cta(smem_u32(&ctl->acc_empty[buf]), 0));
         else mbar_arrive(&ctl->acc_empty[buf]);
       }
-      // 2) registers -> padded shared memory -> global, 64 columns per pass: every store
+      // 2) a contributor other than the owner passes the sum on through the scratch ...
+      if (pass_on) {
+#pragma unroll
+        for (int g = 0; g < BN / 8; ++g)
+          if (row_ok && g * 8 < ncols) sfrag[g * 32] = make_uint4(sum[g * 4 + 0], sum[g * 4 + 1], sum[g * 4 + 2], sum[g * 4 + 3]);
+      }
+      //    ... everything else goes registers -> padded shared memory -> global, 64 columns per pass: every store
       //    instruction writes 4 rows x 128 contiguous bytes.
 #pragma unroll
       for (int pass = 0; pass < BN / 64; ++pass) {
-        if (pass < npass) {
+        if (pass < npass && !pass_on) {
           uint4* srow = reinterpret_cast<uint4*>(stage + lane * kStageRowBytes);
 #pragma unroll
           for (int g = 0; g < 8; ++g)
@@ -1533,7 +1510,7 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   static thread_local GemmParams p;
   // an activation goes with the plain store only (the ring read-modify-write adds partial sums)
   if (L.activation != ACT_NONE && L.epilogue != EPI_STORE) return COMPASS_ERR_INVALID_ARG;
-  if (L.epilogue == EPI_RING_RMW_F32 && L.n_out > 0 && L.sum_ptr[0] == nullptr) return COMPASS_ERR_INVALID_ARG;
+  if (L.epilogue != EPI_STORE && L.ring_scratch == nullptr) return COMPASS_ERR_INVALID_ARG;
   if (L.activation == ACT_SWIGLU && (L.N % 16 != 0 || L.ldo < L.N / 2)) return COMPASS_ERR_INVALID_ARG;
   DeviceInfo* info = nullptr;
   int st = device_info(&info);
@@ -1550,8 +1527,8 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
       return record_cuda_error(cudaErrorUnknown);
   for (int i = 0; i < L.n_out; ++i) {
     p.out[i] = static_cast<__nv_bfloat16*>(L.out_ptr[i]);
-    p.sum[i] = L.sum_ptr[i];
   }
+  p.ring_scratch = static_cast<uint8_t*>(L.ring_scratch);
   p.ldo = L.ldo;
   p.n_blocks = L.n_blocks;
   p.rows_per_block = L.rows_per_block;

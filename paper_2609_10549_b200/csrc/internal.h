@@ -80,7 +80,8 @@ struct GemmParams {
   CUtensorMap b_maps[kMaxP];
   CUtensorMap b_maps_q[kMaxP];   // the same B tensors with boxes of 64 rows (256x128 tiles: 64 B rows per CTA)
   __nv_bfloat16* out[kMaxP];
-  float* sum[kMaxP];       // FP32 running sums, one [rows x N] tensor per output (EPI_RING_RMW_F32 only)
+  uint8_t* ring_scratch;   // ring read-modify-write: running sums, one 128 x 256 fragment after the other in the order
+                           // of the tile counters, each in the order its epilogue warps' lanes hold it
   int64_t ldo;             // output row pitch in elements
   int32_t n_blocks;
   int32_t rows_per_block;
@@ -128,7 +129,7 @@ struct GemmLaunch {
   int64_t a_map_rows[kMaxAMaps] = {};   // rows of A tensor i; 0 = a_rows
   const void* b_ptr[kMaxP];
   void* out_ptr[kMaxP];
-  float* sum_ptr[kMaxP] = {};   // FP32 running sums (EPI_RING_RMW_F32)
+  void* ring_scratch = nullptr;   // running sums of the ring read-modify-write epilogues (one fragment per tile counter)
   int n_a = 0, n_b = 0, n_out = 0;
   int64_t a_rows = 0;      // rows of every A tensor
   int64_t K = 0;           // columns (contraction length) of every A and B tensor

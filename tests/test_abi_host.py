@@ -252,11 +252,16 @@ def test_workspace_sizes():
     assert _codes(ag, api.WS_PUSH) == (api.OK, api.STATUS_BYTES + 256 + 4 * 4096 * 4096 * 2)     # 32 flags + 4 gather buffers
     assert _codes(rs, api.WS_PUSH)[0] == api.ERR_INVALID_ARG
     ring = api.make_problem(OP_GEMM_RS, 8, 8192, 4096, 1376, rs_variant=api.RS_RING_RMW)
-    code, n = _codes(ring)
-    assert code == api.OK and n >= api.STATUS_BYTES + 16 * 4 * 16 * 4
-    # the same with the running sum in FP32 scratch: the counters plus P owners x [M/P x N] floats
+    # 16 partitions x 4 fragments of 128 rows x 16 column tiles: one counter and one BF16 fragment (128 x 256) of
+    # running sum each
+    counters = 16 * 4 * 16
+    assert _codes(ring) == (api.OK, api.STATUS_BYTES + counters * 4 + counters * 128 * 256 * 2)
+    # the same with the running sum in FP32
     ring32 = api.make_problem(OP_GEMM_RS, 8, 8192, 4096, 1376, rs_variant=api.RS_RING_RMW_F32)
-    assert _codes(ring32) == (api.OK, n + 8 * 1024 * 4096 * 4)
+    assert _codes(ring32) == (api.OK, api.STATUS_BYTES + counters * 4 + counters * 128 * 256 * 4)
+    # ragged: 2 partitions x P = 3 of 136 rows (2 fragments) x 520 columns (3 tiles); counters padded to 256 bytes
+    ragged = api.make_problem(OP_GEMM_RS, 3, 3 * 272, 520, 64, rs_variant=api.RS_RING_RMW)
+    assert _codes(ragged) == (api.OK, api.STATUS_BYTES + 256 + 36 * 128 * 256 * 2)
     assert _codes(api.make_problem(OP_GEMM_RS, 8, 8192, 4096, 1376, rs_variant=3))[0] == api.ERR_INVALID_ARG
     plan32 = api.compass_launch_plan(ring32)
     assert [(b.rank, b.step, b.ring) for b in plan32] == [(b.rank, b.step, b.ring) for b in api.compass_launch_plan(ring)]

@@ -305,7 +305,8 @@ def test_small_partitions_ring_rmw_integers_exact_and_counters_return_to_zero():
         assert api.compass_read_status(ws) == (api.OK, 0)
         for o, r in zip(outs, ref):
             assert np.array_equal(ops.bf16_bits_to_f64(o.bits()), r)
-        assert int(ws[api.STATUS_BYTES:].view(torch.int32).abs().sum().item()) == 0
+        n_counters = 2 * w.P * 1 * 3                              # partitions x 128-row fragments x column tiles
+        assert int(ws[api.STATUS_BYTES:api.STATUS_BYTES + 4 * n_counters].view(torch.int32).abs().sum().item()) == 0
 
 
 @pytest.mark.parametrize("op,P,m,N,K,d", [
@@ -646,6 +647,7 @@ def test_ring_rmw_integers_exact_and_counters_return_to_zero():
     pr = gu.problem_of(w, rs_variant=api.RS_RING_RMW)
     A, B = gu.device_inputs(A_bits, B_bits)
     ws = api.alloc_workspace(pr)
+    ws[api.STATUS_BYTES + 256:].fill_(0x7F)     # 48 counters, padded to 256 bytes; behind them garbage (NaN patterns) in the scratch of the running sums
     ref = ops.gemm_rs(A_bits, B_bits)
     for _ in range(2):                                           # the second call reuses the counters
         outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
@@ -653,7 +655,8 @@ def test_ring_rmw_integers_exact_and_counters_return_to_zero():
         assert api.compass_read_status(ws) == (api.OK, 0)
         for o, r in zip(outs, ref):
             assert np.array_equal(ops.bf16_bits_to_f64(o.bits()), r)
-        assert int(ws[api.STATUS_BYTES:].view(torch.int32).abs().sum().item()) == 0
+        n_counters = 2 * w.P * (256 // 128) * 3                   # partitions x 128-row fragments x column tiles
+        assert int(ws[api.STATUS_BYTES:api.STATUS_BYTES + 4 * n_counters].view(torch.int32).abs().sum().item()) == 0
 
 
 def test_config3_ring_rmw_every_element():
