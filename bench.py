@@ -277,16 +277,19 @@ def timing_protocol_report(torch, api, ops_by_name):
 
 
 def rs_variants_report(torch, api, op):
-    """The three GEMM+ReduceScatter forms on the benchmark's GEMM-RS shape, on the device buffers of the timed step:
-    segmented K (the reduction is the accumulator), ring read-modify-write with the running sum in the BF16 output
-    rows, and with the running sum in FP32 scratch.  The three are timed in turn inside one loop (30 rounds, a
+    """The GEMM+ReduceScatter forms on the benchmark's GEMM-RS shape, on the device buffers of the timed step:
+    segmented K (the reduction is the accumulator), ring read-modify-write with a BF16 running sum, with an FP32
+    running sum, and both with two consecutive contributors fused per pass (a ring between P/2 nodes of two ranks
+    each).  They are timed in turn inside one loop (30 rounds, a
     synchronisation after every launch, after a pause that lets the board recover from the sustained loops before it),
     so they are compared at the same board state."""
     stream = torch.cuda.current_stream()
     w = op.w
     runs = {}
-    for name, variant in (("segmented_k", api.RS_SEGMENTED_K), ("ring_rmw", api.RS_RING_RMW), ("ring_rmw_f32", api.RS_RING_RMW_F32)):
-        pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, rs_variant=variant)
+    for name, variant, group in (("segmented_k", api.RS_SEGMENTED_K, 0), ("ring_rmw", api.RS_RING_RMW, 0),
+                                 ("ring_rmw_f32", api.RS_RING_RMW_F32, 0), ("ring_rmw_pairs", api.RS_RING_RMW, 2),
+                                 ("ring_rmw_f32_pairs", api.RS_RING_RMW_F32, 2)):
+        pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, rs_variant=variant, ring_group=group)
         ws = api.alloc_workspace(pr)
         runs[name] = (pr, ws)
     call = lambda name: api.compass_gemm_rs(runs[name][0], op.A, op.B, op.out, runs[name][1], stream)

@@ -136,7 +136,11 @@ typedef struct compass_problem {
   int32_t order;       /* COMPASS_ORDER_* : how the P logical ranks share the one GPU */
   int32_t copy_mode;   /* COMPASS_COPY_* : how compass_decomp moves the AllGather slices */
   int32_t b_layout;    /* COMPASS_B_* : storage of every B_r */
-  int32_t reserved;    /* 0 */
+  int32_t ring_group;  /* COMPASS_RS_RING_RMW / _F32 only, else 0.  0 or 1: every contributor adds its own partial
+                        * to the running sum (what a ring between P GPUs does).  G >= 2, a divisor of P: G consecutive
+                        * contributors of a partition, in ring order, are accumulated in one tile's FP32 accumulator
+                        * first (a ring between P/G nodes of G GPUs each, the node reducing internally): P/G
+                        * read-modify-write passes and P/G roundings instead of P.  G = P is one pass. */
 } compass_problem;
 
 /* One line of the ring chunk schedule (Section III-B).  `part` = rings*chunk +

@@ -108,7 +108,8 @@ def ag_gemm(A: Sequence[np.ndarray], B: Sequence[np.ndarray], table: Optional[np
 
 
 def gemm_rs(A: Sequence[np.ndarray], B: Sequence[np.ndarray], table: Optional[np.ndarray] = None,
-            rings: int = 2, chunks: Optional[Sequence[int]] = None, bf16_hops: bool = False) -> List[np.ndarray]:
+            rings: int = 2, chunks: Optional[Sequence[int]] = None, bf16_hops: bool = False,
+            hop_group: int = 1) -> List[np.ndarray]:
     """Out_c = rows [c*m,(c+1)*m) of sum_q A_q * B_q, reduced along the ring.
 
     For every partition the running sum starts at the rank whose table lists
@@ -118,7 +119,10 @@ def gemm_rs(A: Sequence[np.ndarray], B: Sequence[np.ndarray], table: Optional[np
     ``bf16_hops=False``: the sum itself (FP64), whatever the ring carries.
     ``bf16_hops=True``: the result of a ring whose messages are BF16 -- the sum
     is rounded once per contributor (``hop_in_bf16``), so the result depends on
-    the ORDER of the contributors; the values returned are BF16 values."""
+    the ORDER of the contributors; the values returned are BF16 values.
+    ``hop_group=G`` (a divisor of P): a ring between P/G nodes of G ranks each --
+    G consecutive contributors add up their partials exactly before the node's
+    one hop, so the sum is rounded P/G times."""
     P = len(A)
     M, K = A[0].shape
     N = B[0].shape[0]
@@ -143,7 +147,12 @@ def gemm_rs(A: Sequence[np.ndarray], B: Sequence[np.ndarray], table: Optional[np
             assert int(e[ROW_BEGIN]) == rb and int(e[ROW_COUNT]) == rc and int(e[CHUNK]) == c
             q = int(e[RANK])
             partial = bf16_bits_to_f64(A[q][rb:rb + rc]) @ Bf[q].T
-            running = hop_in_bf16(running, partial) if bf16_hops else running + partial
+            node = partial if int(e[STEP]) % hop_group == 0 else node + partial
+            if not bf16_hops:
+                running = running + partial
+            elif int(e[STEP]) % hop_group == hop_group - 1:
+                running = hop_in_bf16(running, node)
+        assert P % hop_group == 0
         assert int(entries[-1][RANK]) == c, "the running sum must end at the owner"
         if c not in out:
             out[c] = np.full((m, N), np.nan)
@@ -157,7 +166,7 @@ def gemm_rs(A: Sequence[np.ndarray], B: Sequence[np.ndarray], table: Optional[np
 
 
 def gemm_rs_rows(A: Sequence[np.ndarray], B: Sequence[np.ndarray], rows: np.ndarray,
-                 table: Optional[np.ndarray] = None, rings: int = 2, bf16_hops: bool = False):
+                 table: Optional[np.ndarray] = None, rings: int = 2, bf16_hops: bool = False, hop_group: int = 1):
     """GEMM+ReduceScatter restricted to some rows of the reduced [M x N] tensor
     (sorted global row indices), for sampling large cases.  Same ring order as
     ``gemm_rs``.  Returns {owner chunk: (rows inside the owner's block, values)}."""
@@ -182,7 +191,11 @@ def gemm_rs_rows(A: Sequence[np.ndarray], B: Sequence[np.ndarray], rows: np.ndar
         for e in entries:
             q = int(e[RANK])
             partial = bf16_bits_to_f64(A[q][sel]) @ Bf[q].T
-            running = hop_in_bf16(running, partial) if bf16_hops else running + partial
+            node = partial if int(e[STEP]) % hop_group == 0 else node + partial
+            if not bf16_hops:
+                running = running + partial
+            elif int(e[STEP]) % hop_group == hop_group - 1:
+                running = hop_in_bf16(running, node)
         assert int(entries[-1][RANK]) == c
         found.setdefault(c, []).append((sel - c * m, running))
     return {c: (np.concatenate([x[0] for x in v]), np.concatenate([x[1] for x in v])) for c, v in found.items()}

@@ -52,7 +52,7 @@ class Problem(C.Structure):
     _fields_ = [("op", C.c_int32), ("P", C.c_int32), ("rings", C.c_int32), ("d", C.c_int32),
                 ("M", C.c_int64), ("N", C.c_int64), ("K", C.c_int64),
                 ("dtype", C.c_int32), ("rs_variant", C.c_int32), ("order", C.c_int32), ("copy_mode", C.c_int32),
-                ("b_layout", C.c_int32), ("reserved", C.c_int32)]
+                ("b_layout", C.c_int32), ("ring_group", C.c_int32)]
 
 
 class Mlp(C.Structure):
@@ -170,9 +170,9 @@ def _check(status: int, where: str) -> None:
 
 def make_problem(op: int, P: int, M: int, N: int, K: int, rings: int = 2, d: int = 1,
                  rs_variant: int = RS_SEGMENTED_K, dtype: int = DTYPE_BF16, order: int = ORDER_RANK_MAJOR,
-                 copy_mode: int = COPY_KERNEL, b_layout: int = B_NK) -> Problem:
+                 copy_mode: int = COPY_KERNEL, b_layout: int = B_NK, ring_group: int = 0) -> Problem:
     return Problem(op=op, P=P, rings=rings, d=d, M=M, N=N, K=K, dtype=dtype, rs_variant=rs_variant, order=order,
-                   copy_mode=copy_mode, b_layout=b_layout, reserved=0)
+                   copy_mode=copy_mode, b_layout=b_layout, ring_group=ring_group)
 
 
 # ---- host-only calls -------------------------------------------------------------

@@ -31,7 +31,12 @@ int validate_problem(const compass_problem* pr, int want_op, bool need_d) {
   if (pr->op == COMPASS_OP_GEMM_RS && pr->rs_variant != COMPASS_RS_SEGMENTED_K && pr->rs_variant != COMPASS_RS_RING_RMW &&
       pr->rs_variant != COMPASS_RS_RING_RMW_F32)
     return COMPASS_ERR_INVALID_ARG;
-  if ((pr->b_layout != COMPASS_B_NK && pr->b_layout != COMPASS_B_KN) || pr->reserved != 0) return COMPASS_ERR_INVALID_ARG;
+  if (pr->b_layout != COMPASS_B_NK && pr->b_layout != COMPASS_B_KN) return COMPASS_ERR_INVALID_ARG;
+  if (pr->ring_group != 0 && pr->ring_group != 1) {
+    // contributors fused per read-modify-write pass: ring variants only, a divisor of P
+    if (pr->op != COMPASS_OP_GEMM_RS || pr->rs_variant == COMPASS_RS_SEGMENTED_K) return COMPASS_ERR_INVALID_ARG;
+    if (pr->ring_group < 2 || pr->P < 1 || pr->ring_group > pr->P || pr->P % pr->ring_group != 0) return COMPASS_ERR_INVALID_ARG;
+  }
   if (pr->dtype != COMPASS_DTYPE_BF16 || pr->P > COMPASS_MAX_P) return COMPASS_ERR_UNSUPPORTED;
   if (pr->M <= 0 || pr->N <= 0 || pr->K <= 0) return COMPASS_ERR_SHAPE;
   if (pr->M % pr->P != 0 || (pr->M / pr->P) % pr->rings != 0) return COMPASS_ERR_SHAPE;
@@ -179,8 +184,21 @@ void plan_rs_ring(const compass_problem* pr, const compass_sched_entry* table, G
   L->share_run = rings;  // a rank's two ring entries of one step are adjacent and multiply by the same B_rank
   L->epilogue = pr->rs_variant == COMPASS_RS_RING_RMW_F32 ? EPI_RING_RMW_F32 : EPI_RING_RMW;
   L->last_step = P - 1;
+  L->seg_strided = false;
+  L->n_ranks = P;
+  const int G = pr->ring_group > 1 ? pr->ring_group : 1;
+  if (G > 1) {
+    // G consecutive contributors of a partition share a tile: its k-loop runs over their K slices in ring order.
+    // The contributors of a partition follow one another along its ring, so the lead's neighbour (`peer`) gives the
+    // stride between their ranks.
+    L->n_seg = G;
+    L->share_run = 1;
+    L->seg_strided = true;
+    L->last_step = P / G - 1;
+  }
   int n = 0;
-  for (int step = 0; step < P; ++step)
+  bool consistent = true;
+  for (int step = 0; step < P; step += G)
     for (int rank = 0; rank < P; ++rank)        // a rank's entries of one step are adjacent: they share its weight shard in L2
       for (int ring = 0; ring < rings; ++ring) {
         const compass_sched_entry& e = table[(size_t(rank) * P + step) * rings + ring];
@@ -188,13 +206,18 @@ void plan_rs_ring(const compass_problem* pr, const compass_sched_entry* table, G
         std::memset(&b, 0, sizeof(b));
         b.a_map = uint8_t(rank);
         b.b_map = uint8_t(rank);
+        b.seg_stride = uint8_t(G > 1 ? (e.peer - rank + P) % P : 0);
+        for (int i = 1; i < G; ++i) {             // the table must agree: contributor step+i of this partition
+          const int r_i = (rank + i * int(b.seg_stride)) % P;
+          if (table[(size_t(r_i) * P + step + i) * rings + ring].part != e.part) consistent = false;
+        }
         b.a_row0 = e.row_begin;
         b.out_idx = uint8_t(e.chunk);
         b.out_row0 = e.row_begin - e.chunk * int32_t(m);
-        b.step = uint8_t(step);
+        b.step = uint8_t(step / G);
         b.part = uint8_t(e.part);
         if (view) {
-          compass_plan_block& v = view[n];
+          compass_plan_block& v = view[n];      // grouped: the lead contributor's rank and step
           v.rank = rank; v.step = step; v.ring = ring; v.part = e.part;
           v.a_tensor = rank; v.a_row_begin = b.a_row0;
           v.out_tensor = e.chunk; v.out_row_begin = b.out_row0;
@@ -202,7 +225,7 @@ void plan_rs_ring(const compass_problem* pr, const compass_sched_entry* table, G
         }
         ++n;
       }
-  L->n_blocks = n;
+  L->n_blocks = consistent ? n : -1;
 }
 
 int plan_fused(const compass_problem* pr, GemmLaunch* L, compass_plan_block* view) {
@@ -210,9 +233,11 @@ int plan_fused(const compass_problem* pr, GemmLaunch* L, compass_plan_block* vie
   int st = validate_schedule_args(pr->op, pr->P, pr->rings, pr->M);
   if (st != COMPASS_OK) return st;
   build_schedule(pr->op, pr->P, pr->rings, pr->M, table);
+  L->seg_strided = false;
   if (pr->op == COMPASS_OP_AG_GEMM) plan_ag(pr, table, L, view);
   else if (pr->rs_variant == COMPASS_RS_SEGMENTED_K) plan_rs_segmented(pr, table, L, view);
   else plan_rs_ring(pr, table, L, view);
+  if (L->n_blocks < 0) return COMPASS_ERR_UNSUPPORTED;     // (a schedule whose contributors do not follow the ring)
   L->b_mn_major = pr->b_layout == COMPASS_B_KN;
   if (view) {
     const int per_block = tiles_of(L->rows_per_block, gemm_tile_rows(L->mode, L->rows_per_block)) * tiles_of(L->N, BN);
@@ -531,7 +556,8 @@ extern "C" int compass_launch_plan(const compass_problem* pr, compass_plan_block
   int st = validate_problem(pr, -1, false);
   if (st != COMPASS_OK) return st;
   const bool per_entry = pr->op == COMPASS_OP_AG_GEMM || pr->rs_variant != COMPASS_RS_SEGMENTED_K;
-  const size_t n = size_t(pr->rings) * pr->P * (per_entry ? pr->P : 1);
+  const int group = (pr->op == COMPASS_OP_GEMM_RS && pr->ring_group > 1) ? pr->ring_group : 1;   // contributors per block
+  const size_t n = size_t(pr->rings) * pr->P * (per_entry ? pr->P / group : 1);
   *count = n;
   if (out == nullptr) return COMPASS_OK;
   if (capacity < n) return COMPASS_ERR_BUFFER_TOO_SMALL;

@@ -244,7 +244,9 @@ struct StageIter {
     blk = f.blk;
     a_row = b.a_row0 + f.r0;
     b_row = tc.nt * BN + cta_rank * Cfg<kPair>::kBRows;
-    am = (p.n_seg > 1) ? p.seg_rank[tc.blk][seg] : b.a_map;      // segmented K: blocks are never grouped
+    // segmented K (blocks are never grouped): the segment's tensor from the table, or, along a ring, a stride from the lead's
+    am = (p.n_seg > 1) ? (p.seg_strided ? (int(b.a_map) + seg * int(b.seg_stride)) % p.n_ranks : int(p.seg_rank[tc.blk][seg]))
+                       : int(b.a_map);
     bm = (p.n_seg > 1) ? am : b.b_map;                           // the blocks of a group share their B tensor
   }
   __device__ void next(const GemmParams& p) {
@@ -1560,9 +1562,13 @@ int launch_gemm(const GemmLaunch& L, cudaStream_t stream) {
   p.flags = L.flags;
   p.flag_token = L.flag_token;
   for (int b = 0; b < L.n_blocks; ++b) p.blocks[b] = L.blocks[b];
-  if (L.n_seg > 1)
+  p.seg_strided = (L.seg_strided && L.n_seg > 1) ? 1 : 0;
+  p.n_ranks = L.n_ranks > 0 ? L.n_ranks : 1;
+  if (L.n_seg > 1 && !p.seg_strided) {
+    if (L.n_blocks > kMaxSegBlocks) return COMPASS_ERR_UNSUPPORTED;
     for (int b = 0; b < L.n_blocks; ++b)
       for (int s = 0; s < L.n_seg; ++s) p.seg_rank[b][s] = L.seg_rank[b][s];
+  }
 
   if (p.total_tiles <= 0) return COMPASS_OK;
   const bool mixed = tiling.mixed != 0;

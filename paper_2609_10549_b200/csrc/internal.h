@@ -56,7 +56,7 @@ struct BlockDesc {
   uint8_t out_idx;    // index of the output pointer
   uint8_t step;       // schedule step (ring read-modify-write: contributor index)
   uint8_t part;       // schedule partition id
-  uint8_t pad;
+  uint8_t seg_stride; // strided segments (GemmParams.seg_strided): segment s reads tensor (a_map + s * seg_stride) mod n_ranks
   uint16_t flag1;     // 1 + index of the readiness flag the block's A rows wait for (0 = always ready)
 };
 
@@ -120,6 +120,8 @@ struct GemmParams {
   const uint32_t* flags;   // readiness flags (push variant), else nullptr
   uint32_t flag_token;     // a flag is up once it holds a value >= this
   uint8_t seg_rank[kMaxSegBlocks][kMaxP];   // segmented-K: tensor index of segment s of block b
+  int32_t seg_strided;     // 1: the segments' tensors follow BlockDesc.a_map and seg_stride instead of seg_rank
+  int32_t n_ranks;
   BlockDesc blocks[kMaxBlocks];
 };
 
@@ -151,6 +153,8 @@ struct GemmLaunch {
   int n_blocks = 0;
   BlockDesc blocks[kMaxBlocks];
   uint8_t seg_rank[kMaxSegBlocks][kMaxP];
+  bool seg_strided = false;   // segments by BlockDesc.a_map / seg_stride (grouped ring read-modify-write) instead of seg_rank
+  int n_ranks = 0;
   StatusBlock* status = nullptr;
   int32_t* tile_counters = nullptr;
   const uint32_t* flags = nullptr;

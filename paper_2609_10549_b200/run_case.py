@@ -32,6 +32,7 @@ def main():
     ap.add_argument("--K", type=int, required=True)
     ap.add_argument("--d", type=int, default=1)
     ap.add_argument("--rings", type=int, default=2)
+    ap.add_argument("--ring-group", type=int, default=0, help="ring / ring32: contributors fused per read-modify-write pass")
     ap.add_argument("--order", choices=["rank", "step"], default="rank")
     ap.add_argument("--layout", choices=["nk", "kn"], default="nk")
     ap.add_argument("--iters", type=int, default=20)
@@ -62,7 +63,7 @@ def main():
     pr = api.make_problem(op, w.P, w.M, w.N, w.K, rings=args.rings, d=args.d,
                           rs_variant={"ring": api.RS_RING_RMW, "ring32": api.RS_RING_RMW_F32}.get(args.variant, api.RS_SEGMENTED_K),
                           order=api.ORDER_RANK_MAJOR if args.order == "rank" else api.ORDER_STEP_MAJOR,
-                          b_layout=api.B_NK if args.layout == "nk" else api.B_KN)
+                          b_layout=api.B_NK if args.layout == "nk" else api.B_KN, ring_group=args.ring_group)
     stream = torch.cuda.current_stream()
     side = torch.cuda.Stream()
     if args.variant in ("fused", "ring", "ring32"):
@@ -104,7 +105,7 @@ def main():
                           "gbs_median": nbytes / (med * 1e-3) / 1e9}), flush=True)
         return
     print(json.dumps({
-        "op": args.op, "variant": args.variant, "P": w.P, "M": w.M, "N": w.N, "K": w.K, "d": args.d, "rings": args.rings,
+        "op": args.op, "variant": args.variant, "P": w.P, "M": w.M, "N": w.N, "K": w.K, "d": args.d, "rings": args.rings, "ring_group": args.ring_group,
         "order": args.order, "layout": args.layout, "iters": args.iters,
         "ms_median": med, "ms_best": float(np.min(ts)), "tflops_median": w.flops / (med * 1e-3) / 1e12,
         "tflops_best": w.flops / (float(np.min(ts)) * 1e-3) / 1e12,

@@ -222,9 +222,14 @@ def test_problem_validation_codes():
     assert _codes(api.make_problem(**{**ok, "op": 9}))[0] == api.ERR_INVALID_ARG
     assert _codes(api.make_problem(**{**ok, "b_layout": api.B_KN}))[0] == api.OK
     assert _codes(api.make_problem(**{**ok, "b_layout": 2}))[0] == api.ERR_INVALID_ARG
-    nonzero_reserved = api.make_problem(**ok)
-    nonzero_reserved.reserved = 1
-    assert _codes(nonzero_reserved)[0] == api.ERR_INVALID_ARG
+    # contributors fused per read-modify-write pass: ring variants of GEMM+ReduceScatter only, a divisor of P
+    assert _codes(api.make_problem(**ok, ring_group=2))[0] == api.ERR_INVALID_ARG
+    rs = dict(op=OP_GEMM_RS, P=8, M=8192, N=4096, K=1376)
+    assert _codes(api.make_problem(**rs, ring_group=1))[0] == api.OK
+    assert _codes(api.make_problem(**rs, ring_group=2))[0] == api.ERR_INVALID_ARG                   # segmented K
+    for variant in (api.RS_RING_RMW, api.RS_RING_RMW_F32):
+        assert [_codes(api.make_problem(**rs, rs_variant=variant, ring_group=g))[0] for g in (0, 1, 2, 4, 8)] == [api.OK] * 5
+        assert [_codes(api.make_problem(**rs, rs_variant=variant, ring_group=g))[0] for g in (-1, 3, 16)] == [api.ERR_INVALID_ARG] * 3
     assert _codes(api.make_problem(**{**ok, "P": 0}))[0] == api.ERR_INVALID_ARG
     assert _codes(api.make_problem(**ok, rings=3))[0] == api.ERR_INVALID_ARG
     assert _codes(api.make_problem(**{**ok, "P": 32, "M": 4096}))[0] == api.ERR_UNSUPPORTED
@@ -346,3 +351,17 @@ def test_rs_launch_plans(P, rings):
     for (part, step), i in pos_of.items():
         if step > 0:
             assert pos_of[(part, step - 1)] < i
+    # groups of G contributors: one block per (partition, group), named after the group's first contributor
+    who = {(int(e[3]), int(e[1])): int(e[0]) for e in table}                # (part, step) -> rank
+    for G in [g for g in (2, 4, 8) if P % g == 0]:
+        grouped = api.compass_launch_plan(api.make_problem(OP_GEMM_RS, P, M, N, K, rings=rings, rs_variant=api.RS_RING_RMW,
+                                                           ring_group=G))
+        assert len(grouped) == len(table) // G
+        assert sorted((b.part, b.step) for b in grouped) == sorted((part, s) for part in range(rings * P) for s in range(0, P, G))
+        for i, b in enumerate(grouped):
+            assert b.rank == who[(b.part, b.step)] and b.a_tensor == b.rank
+            assert b.out_tensor == b.part // rings and b.rows == m // rings
+        pos_of = {(b.part, b.step): i for i, b in enumerate(grouped)}
+        for (part, step), i in pos_of.items():
+            if step > 0:
+                assert pos_of[(part, step - G)] < i

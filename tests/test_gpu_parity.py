@@ -667,6 +667,81 @@ def test_config3_ring_rmw_every_element():
     check_every_element(w, outs, f"{w.name} ring-RMW", ring_rmw=True)
 
 
+# ---- ring read-modify-write with G consecutive contributors fused per pass (ring_group) --------------------------
+
+def run_ring_grouped(w, A_bits, B_bits, G, rings=2, rs_variant=api.RS_RING_RMW, calls=1):
+    pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, rings=rings, rs_variant=rs_variant, ring_group=G)
+    A, B = gu.device_inputs(A_bits, B_bits)
+    ws = api.alloc_workspace(pr)
+    for _ in range(calls):
+        outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+        api.compass_gemm_rs(pr, A, B, [o.view for o in outs], ws)
+        assert api.compass_read_status(ws) == (api.OK, 0)
+        assert all(o.guards_intact() for o in outs)
+    return [o.bits() for o in outs], ws
+
+
+def check_ring_grouped(outs, A_bits, B_bits, rings, G, what, exact=None):
+    """P/G roundings: held against the ring between P/G nodes computed hop by hop (the oracle's hop_group), with
+    the limits of that many roundings against the exact sum."""
+    P, K = len(A_bits), A_bits[0].shape[1]
+    exact = ops.gemm_rs(A_bits, B_bits, rings=rings) if exact is None else exact
+    hops = ops.gemm_rs(A_bits, B_bits, rings=rings, bf16_hops=True, hop_group=G)
+    for r in range(P):
+        rep = compare.check_bf16_ring(outs[r], exact[r], hops[r], P // G, K * G)
+        assert rep.ok, f"{what} G={G} rank {r}: {rep}"
+
+
+@pytest.mark.parametrize("P,m,N,K,rings,G", [
+    (2, 512, 520, 200, 2, 2), (4, 512, 520, 200, 2, 2), (4, 512, 520, 200, 2, 4), (8, 256, 264, 72, 2, 2),
+    (8, 256, 264, 72, 1, 4), (8, 128, 264, 136, 2, 2), (8, 80, 200, 72, 2, 8), (6, 272, 392, 456, 2, 3),
+    (16, 128, 264, 72, 2, 4), (4, 1024, 776, 344, 1, 2),
+])
+def test_ring_grouped_small_shapes(P, m, N, K, rings, G):
+    w = small(wl.OP_GEMM_RS, P, m, N, K, dist=0.05)
+    A, B = wl.make_inputs(w)
+    exact = ops.gemm_rs(A, B, rings=rings)
+    outs, _ = run_ring_grouped(w, A, B, G, rings=rings)
+    check_ring_grouped(outs, A, B, rings, G, w.name, exact=exact)
+    outs, _ = run_ring_grouped(w, A, B, G, rings=rings, rs_variant=api.RS_RING_RMW_F32)
+    check_all(outs, exact, f"{w.name} FP32 sum G={G}")
+
+
+def test_ring_grouped_integers_exact_and_counters_return_to_zero():
+    w = wl.Workload("ints-ring-grouped", wl.OP_GEMM_RS, P=4, M=4 * 512, N=520, K=64)
+    A_bits, B_bits = wl.make_structured_inputs(w, "index")
+    ref = ops.gemm_rs(A_bits, B_bits)
+    n_counters = 2 * w.P * (256 // 128) * 3
+    for G in (2, 4):
+        for variant in (api.RS_RING_RMW, api.RS_RING_RMW_F32):
+            outs, ws = run_ring_grouped(w, A_bits, B_bits, G, rs_variant=variant, calls=2)
+            for o, r in zip(outs, ref):
+                assert np.array_equal(ops.bf16_bits_to_f64(o), r)
+            assert int(ws[api.STATUS_BYTES:api.STATUS_BYTES + 4 * n_counters].view(torch.int32).abs().sum().item()) == 0
+
+
+def test_ring_group_of_all_contributors_equals_segmented_k():
+    """G = P: one pass, the k-loop over all P slices in ring order -- the segmented-K kernel's arithmetic."""
+    w = small(wl.OP_GEMM_RS, 4, 512, 520, 200, dist=0.05)
+    A, B = wl.make_inputs(w)
+    seg, status, guards = gu.run_fused(w, A, B)
+    assert status == (api.OK, 0) and guards
+    outs, _ = run_ring_grouped(w, A, B, 4)
+    for x, y in zip(outs, seg):
+        assert np.array_equal(x, y)
+
+
+def test_config3_ring_grouped_every_element():
+    w = wl.C3_RS
+    A, B = _inputs(w)
+    outs, _ = run_ring_grouped(w, A, B, 2)
+    for c in range(w.P):
+        ref = _reference(w, c, True)
+        (hops,) = ops.gemm_rs(A, B, chunks=[c], bf16_hops=True, hop_group=2)
+        rep = compare.check_bf16_ring(outs[c], ref, hops, w.P // 2, w.K * 2)
+        assert rep.ok, f"chunk {c}: {rep}"
+
+
 # ---- ring read-modify-write with the running sum in FP32 scratch: one rounding, whatever P ------------------------------
 
 @pytest.mark.parametrize("P,m,N,K,rings", RS_SHAPES + [(16, 128, 264, 72, 2), (16, 64, 520, 200, 1), (8, 384, 776, 72, 2)])

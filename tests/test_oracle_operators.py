@@ -301,3 +301,28 @@ def test_rule_for_a_bf16_ring_tells_the_order_of_the_contributors():
         assert not wrong.ok and wrong.identical < 0.95 and wrong.exact.violations == 0
         once = compare.check_bf16_ring(to_bits(exact[c]), exact[c], hops[c], 8, 40)
         assert not once.ok and once.exact.ok
+
+
+def test_bf16_hops_in_groups_round_once_per_group():
+    """Forward ring, P = 4, one row per chunk; chunk 0's contributors are ranks 1, 2, 3, 0.  With 256, 1, 1, 1:
+    hop by hop 256 + 1 -> 256 three times; in groups of two (256 + 1 = 257 -> 256, then 1 + 1 = 2 added: 258);
+    in one group of four the exact 259 rounds to 260 (tie to even).  Groups of one are the plain hops, and without
+    BF16 hops the grouping changes nothing."""
+    P = 4
+    values = np.zeros((P, P))
+    values[1][0], values[2][0], values[3][0], values[0][0] = 256.0, 1.0, 1.0, 1.0
+    A, B = scalar_shards(P, 1, values)
+    got = {g: float(ops.gemm_rs(A, B, rings=1, bf16_hops=True, hop_group=g)[0][0, 0]) for g in (1, 2, 4)}
+    assert got == {1: 256.0, 2: 258.0, 4: 260.0}
+    assert float(ops.gemm_rs(A, B, rings=1, hop_group=2)[0][0, 0]) == 259.0
+    w, A, B = tiny(OP_GEMM_RS, 8, 8 * 16, 24, 40, seed=9)
+    for g in (2, 4, 8):
+        grouped = ops.gemm_rs(A, B, bf16_hops=True, hop_group=g)
+        rows = np.array([0, 5, 17, 40, 127])
+        sampled = ops.gemm_rs_rows(A, B, rows, bf16_hops=True, hop_group=g)
+        for c, (local, vals) in sampled.items():
+            assert np.array_equal(vals, grouped[c][local])
+    once = ops.gemm_rs(A, B, bf16_hops=True, hop_group=8)                      # one rounding of the FP32 sum
+    exact = ops.gemm_rs(A, B)
+    for o, e in zip(once, exact):
+        assert np.array_equal(o, ops.fp32_to_bf16_rne(e.astype(np.float32)))
