@@ -1029,6 +1029,30 @@ def _random_rs_cases(n, seed):
     return [c for c in _random_cases(4 * n, seed) if c[0] == wl.OP_GEMM_RS][:n]
 
 
+@pytest.mark.parametrize("op,P,m,N,K,rings,order,variant,layout", _random_rs_cases(16, seed=78))
+def test_random_shapes_ring_grouped(op, P, m, N, K, rings, order, variant, layout):
+    """The group size drawn from the divisors of P (above 1), weight layout and running-sum type from the case."""
+    divisors = [g for g in range(2, P + 1) if P % g == 0]
+    if not divisors:
+        pytest.skip("P = 1 has no group")
+    G = divisors[(m + N + K) % len(divisors)]
+    w = small(op, P, m, N, K, seed=P + m + N + K + 2, dist=0.1)
+    A_bits, B_bits = wl.make_inputs(w)
+    rs_variant = api.RS_RING_RMW_F32 if variant else api.RS_RING_RMW
+    pr = api.make_problem(w.op, w.P, w.M, w.N, w.K, rings=rings, rs_variant=rs_variant, b_layout=layout, ring_group=G)
+    A = [api.to_device(a) for a in A_bits]
+    B = [api.to_device(np.ascontiguousarray(b.T) if layout == api.B_KN else b) for b in B_bits]
+    outs = [gu.Guarded(*w.out_shape) for _ in range(w.P)]
+    ws = api.alloc_workspace(pr)
+    api.compass_gemm_rs(pr, A, B, [o.view for o in outs], ws)
+    assert api.compass_read_status(ws) == (api.OK, 0)
+    assert all(o.guards_intact() for o in outs)
+    if rs_variant == api.RS_RING_RMW_F32:
+        check_all([o.bits() for o in outs], ops.gemm_rs(A_bits, B_bits, rings=rings), f"{w.name} G={G}")
+    else:
+        check_ring_grouped([o.bits() for o in outs], A_bits, B_bits, rings, G, w.name)
+
+
 @pytest.mark.parametrize("op,P,m,N,K,rings,order,variant,layout", _random_rs_cases(12, seed=77))
 def test_random_shapes_ring_f32(op, P, m, N, K, rings, order, variant, layout):
     w = small(op, P, m, N, K, seed=P + m + N + K + 1, dist=0.1)
