@@ -408,7 +408,10 @@ typedef struct compass_tile_counts {
   int32_t total_tiles;
 } compass_tile_counts;
 int compass_tile_plan(const compass_problem* problem, int decomposed, int cta_pairs, compass_tile_counts* out);
-/* The blocks of the fused launch for this problem, in launch order. */
+/* The blocks of the fused launch for this problem, in launch order.  With
+ * problem->ring_group = G > 1 a block stands for G consecutive contributors of a
+ * partition and carries the rank and the step of the first of them; there are
+ * rings * P * P / G blocks. */
 int compass_launch_plan(const compass_problem* problem, compass_plan_block* out, size_t capacity, size_t* count);
 /* End-to-end convenience with HOST tensors: copies A and B (host pointers,
  * pinned memory recommended) into `staging` (device, >= *staging_bytes_needed),
